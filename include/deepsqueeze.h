@@ -1,0 +1,198 @@
+/*
+ * deepsqueeze.h -- C ABI of the DeepSqueeze node-update library for one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library runs one iteration of Algorithm 1 ("DeepSqueeze", error-
+ * compensated compressed decentralized SGD) for n simulated nodes that are
+ * stored as the rows of device arrays on ONE GPU:
+ *
+ *     g_i      = stochastic gradient of f_i at x_i                (Algorithm 1, gradient step)
+ *     v_i      = x_i - gamma g_i + delta_i                        (error-compensated variable)
+ *     C[v_i], delta_i <- v_i - C[v_i]                             (compression step)
+ *     x_i     <- x_i - gamma g_i + eta sum_{j in N(i)} (W_ij - I_ij) C[v_j]   (local update;
+ *                i itself belongs to N(i); Section 3 gives the same rule in matrix form)
+ *
+ * "Send" and "receive" of Algorithm 1 are a read of the packed codes that all
+ * nodes of the simulation share on the device.
+ *
+ * Conventions
+ *   - All arrays are row-major [n][ld] binary32 with a common row pitch ld
+ *     (elements), ld >= N, ld a multiple of 4, base pointers 16-byte aligned.
+ *     Columns N..ld-1 are padding: read, never changed.
+ *   - Pointers are DEVICE pointers unless the comment says "host".
+ *   - The caller owns every buffer, the workspace included; the library
+ *     allocates no device memory.  x and delta are updated in place.
+ *   - Every call returns a ds_status; nothing throws.  ds_step only enqueues
+ *     work on the given stream and reports argument and launch errors.
+ *   - One ds_ctx must not be used from two streams at once (the steps share
+ *     the workspace).
+ */
+#ifndef DEEPSQUEEZE_H
+#define DEEPSQUEEZE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ds_ctx ds_ctx;   /* opaque; created by ds_init, freed by ds_destroy */
+
+typedef enum {
+    DS_OK = 0,
+    DS_ERR_NULL = 1,             /* a required pointer is NULL */
+    DS_ERR_ARG = 2,              /* a size or scalar argument is out of range */
+    DS_ERR_GRAPH = 3,            /* CSR malformed: row_ptr not monotone, column out of range, unsorted or duplicate */
+    DS_ERR_W_NOT_SYMMETRIC = 4,  /* |W_ij - W_ji| > 1e-6, or the pattern itself is not symmetric */
+    DS_ERR_W_NOT_STOCHASTIC = 5, /* a row sum differs from 1 by more than 1e-6, or a weight is negative */
+    DS_ERR_NO_SELF_LOOP = 6,     /* some node is not its own neighbour */
+    DS_ERR_ALIGN = 7,            /* pointer not 16-byte aligned, or pitch not a multiple of 4 */
+    DS_ERR_WORKSPACE = 8,        /* workspace smaller than ds_workspace_size() */
+    DS_ERR_UNSUPPORTED = 9,      /* combination not implemented (e.g. bits not in {1,2,4,8}) */
+    DS_ERR_CUDA = 10             /* a CUDA runtime call failed (no device, launch error, ...) */
+} ds_status;
+
+/* Node graph in CSR form, HOST memory: row i lists N(i) in ascending order
+ * and contains i itself (Algorithm 1, receive step: "i in N(i)"). */
+typedef struct {
+    int32_t n;
+    const int32_t *row_ptr;     /* host, n+1 entries, row_ptr[0] = 0 */
+    const int32_t *col_idx;     /* host, row_ptr[n] entries */
+} ds_graph;
+
+/* Compressor C_omega (Algorithm 1, compression step; Section 5, "Compression":
+ * every element is sent with b bits plus one scalar per tensor).
+ *   DS_COMP_IDENTITY             C[v] = v (D-PSGD, Section 3.2); the "codes" are the
+ *                                bit patterns of v, 32 bits per element; bits is ignored.
+ *   DS_COMP_SIGN1_L1             one bit per element: bit = (v >= 0); C = +s / -s with
+ *                                s = (sum |v|)/m over the chunk (binary64 sum); bits must be 1.
+ *   DS_COMP_UNIFORM_STOCH_MAXABS b in {1,2,4,8} bits: 2^b levels evenly spaced on
+ *                                [-s, s], s = max |v| over the chunk, stochastic rounding
+ *                                with a Philox4x32-10 stream; unbiased.
+ * chunk: elements per scale, a multiple of 32; 0 = one scale per node. */
+typedef enum {
+    DS_COMP_IDENTITY = 0,
+    DS_COMP_SIGN1_L1 = 1,
+    DS_COMP_UNIFORM_STOCH_MAXABS = 2
+} ds_comp_kind;
+
+typedef struct {
+    int32_t kind;               /* ds_comp_kind */
+    int32_t bits;
+    int64_t chunk;
+} ds_compressor;
+
+/* Stochastic gradient of the synthetic objective (Eq. 1 with
+ * f_i(x) = 1/2 sum_k a_ik (x_k - c_ik)^2):  g_ik = a_ik (x_ik - c_ik) + sigma z_ik,
+ * z drawn inside the kernel from Philox4x32-10 keyed by (seed, node, step, index). */
+typedef enum {
+    DS_NOISE_NONE = 0,
+    DS_NOISE_GAUSS = 1,         /* standard normal (Box-Muller) */
+    DS_NOISE_STUDENT_T3 = 2     /* Student t, 3 degrees of freedom, not re-normalised */
+} ds_noise_kind;
+
+typedef struct {
+    const float *a;             /* device [n][ld] */
+    const float *c;             /* device [n][ld] */
+    float sigma;
+    int32_t noise;              /* ds_noise_kind */
+} ds_grad_params;
+
+typedef struct {
+    float gamma;                /* learning rate (multiplies g only) */
+    float eta;                  /* averaging rate (multiplies the whole neighbour sum) */
+} ds_hparams;
+
+/* How a step is executed.
+ *   DS_PATH_FUSED  one kernel: a thread block owns one chunk column of ALL nodes, keeps
+ *                  x - gamma g in registers and the column's codes in shared memory, and
+ *                  mixes without re-reading anything from global memory.
+ *   DS_PATH_SPLIT  two kernels: compress (x - gamma g written into x, codes to the
+ *                  workspace), then mix (codes re-read).  Works for every shape.
+ *   DS_PATH_AUTO   fused when the shape allows it, else split. */
+typedef enum { DS_PATH_AUTO = 0, DS_PATH_FUSED = 1, DS_PATH_SPLIT = 2 } ds_path;
+
+typedef struct {
+    int32_t path;               /* ds_path actually used by ds_step */
+    int32_t launches_per_step;  /* kernels enqueued by one ds_step */
+    int32_t elems_per_lane;     /* consecutive elements a lane owns within a chunk */
+    int32_t warps_per_chunk;    /* warps that share one (node, chunk) */
+    int32_t block_threads;      /* threads per block of the main kernel */
+    int32_t grid_blocks;        /* blocks of the main kernel */
+    int64_t chunks_per_row;     /* M = ceil(N / chunk) */
+    int64_t code_words_per_row; /* ceil(N * code_bits / 32) */
+} ds_info;
+
+/* Bytes of device workspace ds_init needs for this shape (host-only call;
+ * returns 0 for invalid arguments).  nnz = row_ptr[n]. */
+size_t ds_workspace_size(int32_t n, int64_t N, const ds_compressor *comp, int32_t nnz);
+
+/* Validate the graph and W (Assumption 1: W symmetric, doubly stochastic;
+ * Algorithm 1: every node its own neighbour), copy them to the workspace and
+ * create a context.
+ *   graph      host CSR (see ds_graph)
+ *   W          host, one binary32 weight per CSR entry, in CSR order
+ *   n, N, ld   nodes, parameters per node, row pitch (elements)
+ *   comp       compressor
+ *   workspace  device memory, 256-byte aligned, at least ds_workspace_size() bytes;
+ *              must stay valid until ds_destroy
+ * All validation happens before the first CUDA call, so argument errors are
+ * reported on machines without a GPU.  On failure *out is NULL. */
+ds_status ds_init(ds_ctx **out, const ds_graph *graph, const float *W,
+                  int32_t n, int64_t N, int64_t ld, const ds_compressor *comp,
+                  void *workspace, size_t workspace_bytes);
+
+/* One iteration of Algorithm 1 for all nodes, enqueued on `cuda_stream`
+ * (a cudaStream_t; NULL = default stream).
+ *   x, delta   device [n][ld], updated in place
+ *   gp         gradient data (a, c device [n][ld]) and noise
+ *   hp         gamma, eta of this iteration (the paper decays the learning rate)
+ *   seed,step  select the random streams; step < 2^56.  The same
+ *              (seed, step) always reproduces the same iteration. */
+ds_status ds_step(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
+                  const ds_hparams *hp, uint64_t seed, uint64_t step, void *cuda_stream);
+
+/* Same iteration for HOST buffers: copies x, delta, a, c (host, [n][ld]) into
+ * the caller's device staging arrays, runs ds_step, and copies x and delta
+ * back, all enqueued on `cuda_stream`; the caller synchronises the stream
+ * before reading the results.  Host buffers should be page-locked for the
+ * copies to be asynchronous.  dev_* are device [n][ld] arrays owned by the
+ * caller. */
+ds_status ds_step_host(ds_ctx *ctx, float *x_host, float *delta_host,
+                       const float *a_host, const float *c_host,
+                       float sigma, int32_t noise, const ds_hparams *hp,
+                       uint64_t seed, uint64_t step,
+                       float *dev_x, float *dev_delta, float *dev_a, float *dev_c,
+                       void *cuda_stream);
+
+/* Device pointers to what the nodes "sent" in the last step (Algorithm 1, send
+ * step): packed codes [n][*code_pitch_words] (element k of a node occupies
+ * bits (k*b)%32 .. of word (k*b)/32, little-endian) and scales
+ * [n][*scales_pitch], one per (node, chunk).  Valid until the next ds_step;
+ * no copy is made. */
+ds_status ds_codes(ds_ctx *ctx, const uint32_t **codes, int64_t *code_pitch_words,
+                   const float **scales, int64_t *scales_pitch);
+
+/* Choose the execution path (default DS_PATH_AUTO).  DS_ERR_UNSUPPORTED if
+ * DS_PATH_FUSED is asked for a shape it cannot take. */
+ds_status ds_set_path(ds_ctx *ctx, int32_t path);
+
+/* Launch geometry of the current path (host-only). */
+ds_status ds_get_info(const ds_ctx *ctx, ds_info *info);
+
+/* Diagnostics: write the random streams the kernels draw from, one value per
+ * element, out[node][k] for k < N (device, [n][ld_out]).  which = 0: unit
+ * gradient noise z of kind `noise`; which = 1: the rounding uniforms in
+ * [0, 1).  Lets a caller check stream reproducibility without running a step. */
+ds_status ds_noise(float *out, int32_t n, int64_t N, int64_t ld_out, int32_t which,
+                   int32_t noise, uint64_t seed, uint64_t step, void *cuda_stream);
+
+void ds_destroy(ds_ctx *ctx);
+
+const char *ds_strerror(ds_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEEPSQUEEZE_H */

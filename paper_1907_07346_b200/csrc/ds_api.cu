@@ -1,0 +1,392 @@
+// Host side of the DeepSqueeze C ABI: argument and graph validation,
+// workspace carving, launch planning and dispatch.  See include/deepsqueeze.h.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/deepsqueeze.h"
+#include "ds_column_kernel.cuh"
+
+using namespace ds;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int64_t kPerNodeTile = 512;   // tile width when one scale covers a node
+constexpr int kMaxSmem = 227 * 1024;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int64_t round_up64(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+struct Shape {
+    int code;             // CODE_*
+    int code_bits;
+    int64_t chunk;        // elements per scale (N when one per node)
+    int64_t M;            // scales per row
+    int64_t tile;         // column tile of the kernels
+    int64_t tiles;
+    bool per_node;        // scale computed by a separate reduction
+    int64_t code_words, code_pitch, scales_pitch;
+};
+
+struct WsLayout {
+    size_t codes, scales, partials, row_ptr, col_idx, wprime, lut, total;
+};
+
+bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
+    if (!comp || n < 1 || N < 1) return false;
+    switch (comp->kind) {
+        case DS_COMP_IDENTITY: sh->code = CODE_ID32; break;
+        case DS_COMP_SIGN1_L1:
+            if (comp->bits != 1) return false;
+            sh->code = CODE_SIGN;
+            break;
+        case DS_COMP_UNIFORM_STOCH_MAXABS:
+            if (comp->bits == 1) sh->code = CODE_U1;
+            else if (comp->bits == 2) sh->code = CODE_U2;
+            else if (comp->bits == 4) sh->code = CODE_U4;
+            else if (comp->bits == 8) sh->code = CODE_U8;
+            else return false;
+            break;
+        default: return false;
+    }
+    if (comp->chunk < 0 || (comp->chunk % 32) != 0) return false;
+    sh->code_bits = code_bits_of(sh->code);
+    const bool identity = (sh->code == CODE_ID32);
+    sh->per_node = (comp->chunk == 0) && !identity;
+    sh->chunk = (comp->chunk == 0) ? N : comp->chunk;
+    sh->M = identity ? 0 : (N + sh->chunk - 1) / sh->chunk;
+    sh->tile = (comp->chunk == 0) ? kPerNodeTile : comp->chunk;
+    sh->tiles = (N + sh->tile - 1) / sh->tile;
+    sh->code_words = (N * sh->code_bits + 31) / 32;
+    sh->code_pitch = round_up64(sh->code_words, 4);
+    sh->scales_pitch = round_up64(std::max<int64_t>(sh->M, 1), 4);
+    return true;
+}
+
+WsLayout make_ws(int32_t n, int32_t nnz, const Shape& sh) {
+    WsLayout w;
+    size_t off = 0;
+    w.codes = off;    off = align_up(off + (size_t)n * (size_t)sh.code_pitch * 4, kAlign);
+    w.scales = off;   off = align_up(off + (size_t)n * (size_t)sh.scales_pitch * 4, kAlign);
+    w.partials = off; off = align_up(off + (sh.per_node ? (size_t)n * (size_t)sh.tiles * 8 : 0), kAlign);
+    w.row_ptr = off;  off = align_up(off + (size_t)(n + 1) * 4, kAlign);
+    w.col_idx = off;  off = align_up(off + (size_t)nnz * 4, kAlign);
+    w.wprime = off;   off = align_up(off + (size_t)nnz * 4, kAlign);
+    w.lut = off;      off = align_up(off + 256 * 4, kAlign);
+    w.total = off;
+    return w;
+}
+
+struct Plan {
+    bool ok = false;
+    int elems_per_lane = 0;
+    int warps_per_group = 0;
+    int nodes_per_block = 0;
+    dim3 grid, block;
+    size_t smem = 0;
+};
+
+void pick_lane_shape(int64_t tile, int* E, int* G) {
+    *E = (tile >= 512) ? 16 : (tile >= 256) ? 8 : 4;
+    *G = (int)((tile + 32 * (*E) - 1) / (32 * (*E)));
+}
+
+Plan plan_column(int mode, const Shape& sh, int32_t n, int32_t nnz) {
+    Plan pl;
+    int E, G;
+    pick_lane_shape(sh.tile, &E, &G);
+    pl.elems_per_lane = E;
+    pl.warps_per_group = G;
+    if (G > 32) return pl;
+    int npb;
+    if (mode == MODE_FUSED) {
+        if (sh.code == CODE_ID32) return pl;
+        if ((int64_t)n * G > 32) return pl;
+        npb = n;
+    } else {
+        npb = std::max(1, std::min<int>(n, 8 / G));
+    }
+    pl.nodes_per_block = npb;
+    pl.block = dim3((unsigned)(npb * G * 32));
+    const bool lut = !(sh.code == CODE_SIGN || sh.code == CODE_ID32);
+    pl.smem = smem_layout(mode, sh.code_bits, lut, npb, G, sh.tile, n, nnz).total;
+    if (pl.smem > (size_t)kMaxSmem) return pl;
+    const int64_t gx = std::min<int64_t>(sh.tiles, 0x7fffffff);
+    pl.grid = dim3((unsigned)gx, (unsigned)((n + npb - 1) / npb));
+    pl.ok = true;
+    return pl;
+}
+
+}  // namespace
+
+struct ds_ctx {
+    int32_t n, nnz;
+    int64_t N, ld;
+    ds_compressor comp;
+    Shape sh;
+    WsLayout ws;
+    unsigned char* base;
+    int path_req;
+    Plan fused, compress, reduce;
+};
+
+extern "C" {
+
+const char* ds_strerror(ds_status status) {
+    switch (status) {
+        case DS_OK: return "ok";
+        case DS_ERR_NULL: return "a required pointer is NULL";
+        case DS_ERR_ARG: return "argument out of range";
+        case DS_ERR_GRAPH: return "malformed CSR graph";
+        case DS_ERR_W_NOT_SYMMETRIC: return "W is not symmetric";
+        case DS_ERR_W_NOT_STOCHASTIC: return "W is not (doubly) stochastic";
+        case DS_ERR_NO_SELF_LOOP: return "a node is not its own neighbour";
+        case DS_ERR_ALIGN: return "pointer or pitch misaligned";
+        case DS_ERR_WORKSPACE: return "workspace too small";
+        case DS_ERR_UNSUPPORTED: return "unsupported combination";
+        case DS_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+size_t ds_workspace_size(int32_t n, int64_t N, const ds_compressor* comp, int32_t nnz) {
+    Shape sh;
+    if (nnz < 1 || !make_shape(n, N, comp, &sh)) return 0;
+    return make_ws(n, nnz, sh).total;
+}
+
+ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n, int64_t N,
+                  int64_t ld, const ds_compressor* comp, void* workspace, size_t workspace_bytes) {
+    if (!out) return DS_ERR_NULL;
+    *out = nullptr;
+    if (!graph || !graph->row_ptr || !graph->col_idx || !W || !comp || !workspace) return DS_ERR_NULL;
+    if (n < 1 || N < 1 || N >= ((int64_t)1 << 31) || graph->n != n || ld < N) return DS_ERR_ARG;
+    if ((ld % 4) != 0) return DS_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0) return DS_ERR_ALIGN;
+    if (comp->kind < DS_COMP_IDENTITY || comp->kind > DS_COMP_UNIFORM_STOCH_MAXABS) return DS_ERR_ARG;
+    if (comp->chunk < 0 || (comp->chunk % 32) != 0) return DS_ERR_ARG;
+    Shape sh;
+    if (!make_shape(n, N, comp, &sh)) return DS_ERR_UNSUPPORTED;
+
+    // ---- graph: CSR well formed, sorted, self loop (Algorithm 1: i in N(i)) ----
+    const int32_t* rp = graph->row_ptr;
+    const int32_t* ci = graph->col_idx;
+    if (rp[0] != 0) return DS_ERR_GRAPH;
+    for (int32_t i = 0; i < n; ++i)
+        if (rp[i + 1] < rp[i]) return DS_ERR_GRAPH;
+    const int32_t nnz = rp[n];
+    if (nnz < n) {
+        // fewer entries than nodes: some row cannot hold its diagonal
+        for (int32_t i = 0; i < n; ++i) {
+            bool self = false;
+            for (int32_t e = rp[i]; e < rp[i + 1]; ++e) self = self || (ci[e] == i);
+            if (!self) return DS_ERR_NO_SELF_LOOP;
+        }
+        return DS_ERR_GRAPH;
+    }
+    for (int32_t i = 0; i < n; ++i) {
+        bool self = false;
+        for (int32_t e = rp[i]; e < rp[i + 1]; ++e) {
+            if (ci[e] < 0 || ci[e] >= n) return DS_ERR_GRAPH;
+            if (e > rp[i] && ci[e] <= ci[e - 1]) return DS_ERR_GRAPH;
+            self = self || (ci[e] == i);
+        }
+        if (!self) return DS_ERR_NO_SELF_LOOP;
+    }
+    // ---- W: non-negative, symmetric, rows sum to one (Assumption 1) ----
+    for (int32_t i = 0; i < n; ++i) {
+        double rs = 0.0;
+        for (int32_t e = rp[i]; e < rp[i + 1]; ++e) {
+            const float w = W[e];
+            if (!(w >= 0.0f) || !std::isfinite(w)) return DS_ERR_W_NOT_STOCHASTIC;
+            rs += (double)w;
+            const int32_t j = ci[e];
+            const int32_t* lo = ci + rp[j];
+            const int32_t* hi = ci + rp[j + 1];
+            const int32_t* it = std::lower_bound(lo, hi, i);
+            if (it == hi || *it != i) return DS_ERR_W_NOT_SYMMETRIC;
+            if (std::fabs((double)W[it - ci] - (double)w) > 1e-6) return DS_ERR_W_NOT_SYMMETRIC;
+        }
+        if (std::fabs(rs - 1.0) > 1e-6) return DS_ERR_W_NOT_STOCHASTIC;
+    }
+    const WsLayout ws = make_ws(n, nnz, sh);
+    if (workspace_bytes < ws.total) return DS_ERR_WORKSPACE;
+
+    ds_ctx* ctx = new (std::nothrow) ds_ctx;
+    if (!ctx) return DS_ERR_ARG;
+    ctx->n = n; ctx->nnz = nnz; ctx->N = N; ctx->ld = ld;
+    ctx->comp = *comp; ctx->sh = sh; ctx->ws = ws;
+    ctx->base = static_cast<unsigned char*>(workspace);
+    ctx->path_req = DS_PATH_AUTO;
+    ctx->fused = plan_column(MODE_FUSED, sh, n, nnz);
+    ctx->compress = plan_column(MODE_COMPRESS, sh, n, nnz);
+    ctx->reduce = plan_column(MODE_REDUCE, sh, n, nnz);
+    if (!ctx->compress.ok) { delete ctx; return DS_ERR_UNSUPPORTED; }
+
+    // w'_ij = W_ij - I_ij in binary32; reconstruction levels (2q - L)/L.
+    std::vector<float> wprime((size_t)nnz);
+    for (int32_t i = 0; i < n; ++i)
+        for (int32_t e = rp[i]; e < rp[i + 1]; ++e)
+            wprime[(size_t)e] = W[e] - ((ci[e] == i) ? 1.0f : 0.0f);
+    float lut[256];
+    std::memset(lut, 0, sizeof(lut));
+    if (sh.code != CODE_ID32) {
+        const int L = (1 << sh.code_bits) - 1;
+        for (int q = 0; q <= L; ++q) lut[q] = (float)((double)(2 * q - L) / (double)L);
+    }
+    cudaError_t e = cudaMemcpy(ctx->base + ws.row_ptr, rp, (size_t)(n + 1) * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.col_idx, ci, (size_t)nnz * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.wprime, wprime.data(), (size_t)nnz * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.lut, lut, sizeof(lut), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.codes, 0, ws.scales - ws.codes);
+    if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.scales, 0, ws.partials - ws.scales);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete ctx;
+        return DS_ERR_CUDA;
+    }
+    *out = ctx;
+    return DS_OK;
+}
+
+void ds_destroy(ds_ctx* ctx) { delete ctx; }
+
+static bool use_fused(const ds_ctx* ctx) {
+    if (ctx->path_req == DS_PATH_SPLIT) return false;
+    return ctx->fused.ok;
+}
+
+ds_status ds_set_path(ds_ctx* ctx, int32_t path) {
+    if (!ctx) return DS_ERR_NULL;
+    if (path < DS_PATH_AUTO || path > DS_PATH_SPLIT) return DS_ERR_ARG;
+    if (path == DS_PATH_FUSED && !ctx->fused.ok) return DS_ERR_UNSUPPORTED;
+    ctx->path_req = path;
+    return DS_OK;
+}
+
+ds_status ds_get_info(const ds_ctx* ctx, ds_info* info) {
+    if (!ctx || !info) return DS_ERR_NULL;
+    const bool fused = use_fused(ctx);
+    const Plan& pl = fused ? ctx->fused : ctx->compress;
+    info->path = fused ? DS_PATH_FUSED : DS_PATH_SPLIT;
+    info->launches_per_step = (fused ? 1 : 2) + (ctx->sh.per_node ? 2 : 0);
+    info->elems_per_lane = pl.elems_per_lane;
+    info->warps_per_chunk = pl.warps_per_group;
+    info->block_threads = (int32_t)pl.block.x;
+    info->grid_blocks = (int32_t)(pl.grid.x * pl.grid.y);
+    info->chunks_per_row = ctx->sh.M;
+    info->code_words_per_row = ctx->sh.code_words;
+    return DS_OK;
+}
+
+ds_status ds_codes(ds_ctx* ctx, const uint32_t** codes, int64_t* code_pitch_words,
+                   const float** scales, int64_t* scales_pitch) {
+    if (!ctx || !codes || !code_pitch_words || !scales || !scales_pitch) return DS_ERR_NULL;
+    *codes = reinterpret_cast<const uint32_t*>(ctx->base + ctx->ws.codes);
+    *code_pitch_words = ctx->sh.code_pitch;
+    *scales = reinterpret_cast<const float*>(ctx->base + ctx->ws.scales);
+    *scales_pitch = ctx->sh.scales_pitch;
+    return DS_OK;
+}
+
+ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const ds_hparams* hp,
+                  uint64_t seed, uint64_t step, void* cuda_stream) {
+    if (!ctx || !x || !delta || !gp || !hp || !gp->a || !gp->c) return DS_ERR_NULL;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    if (step >= ((uint64_t)1 << 56)) return DS_ERR_ARG;
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
+                           reinterpret_cast<uintptr_t>(gp->a) | reinterpret_cast<uintptr_t>(gp->c);
+    if ((bits % 16) != 0) return DS_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    StepParams p;
+    p.x = x; p.delta = delta; p.a = gp->a; p.c = gp->c;
+    p.ld = ctx->ld; p.N = ctx->N; p.n = ctx->n; p.nnz = ctx->nnz;
+    p.tile = ctx->sh.tile; p.tiles = ctx->sh.tiles;
+    p.row_ptr = reinterpret_cast<const int32_t*>(ctx->base + ctx->ws.row_ptr);
+    p.col_idx = reinterpret_cast<const int32_t*>(ctx->base + ctx->ws.col_idx);
+    p.wprime = reinterpret_cast<const float*>(ctx->base + ctx->ws.wprime);
+    p.lut = reinterpret_cast<const float*>(ctx->base + ctx->ws.lut);
+    p.codes = reinterpret_cast<uint32_t*>(ctx->base + ctx->ws.codes);
+    p.code_pitch = ctx->sh.code_pitch;
+    p.scales = reinterpret_cast<float*>(ctx->base + ctx->ws.scales);
+    p.scales_pitch = ctx->sh.scales_pitch;
+    p.partials = reinterpret_cast<double*>(ctx->base + ctx->ws.partials);
+    p.sigma = gp->sigma;
+    p.neg_gamma = -hp->gamma;
+    p.eta = hp->eta;
+    p.rs = make_rng_step(seed, step);
+    p.prescaled = ctx->sh.per_node ? 1 : 0;
+
+    auto shape_of = [&](const Plan& pl, int mode) {
+        LaunchShape s;
+        s.code = ctx->sh.code; s.noise = gp->noise; s.elems_per_lane = pl.elems_per_lane;
+        s.mode = mode; s.grid = pl.grid; s.block = pl.block; s.smem = pl.smem;
+        return s;
+    };
+    cudaError_t e = cudaSuccess;
+    if (ctx->sh.per_node) {
+        p.warps_per_group = ctx->reduce.warps_per_group;
+        p.nodes_per_block = ctx->reduce.nodes_per_block;
+        e = launch_column_reduce(shape_of(ctx->reduce, MODE_REDUCE), p, stream);
+        if (e == cudaSuccess) e = launch_finalize_scales(p, ctx->sh.code, stream);
+    }
+    if (e == cudaSuccess) {
+        if (use_fused(ctx)) {
+            p.warps_per_group = ctx->fused.warps_per_group;
+            p.nodes_per_block = ctx->fused.nodes_per_block;
+            e = launch_column_fused(shape_of(ctx->fused, MODE_FUSED), p, stream);
+        } else {
+            p.warps_per_group = ctx->compress.warps_per_group;
+            p.nodes_per_block = ctx->compress.nodes_per_block;
+            e = launch_column_compress(shape_of(ctx->compress, MODE_COMPRESS), p, stream);
+            if (e == cudaSuccess) e = launch_mix_kernel(p, ctx->sh.code, stream);
+        }
+    }
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DS_ERR_CUDA;
+    }
+    return DS_OK;
+}
+
+ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const float* a_host,
+                       const float* c_host, float sigma, int32_t noise, const ds_hparams* hp,
+                       uint64_t seed, uint64_t step, float* dev_x, float* dev_delta, float* dev_a,
+                       float* dev_c, void* cuda_stream) {
+    if (!ctx || !x_host || !delta_host || !a_host || !c_host || !hp || !dev_x || !dev_delta ||
+        !dev_a || !dev_c)
+        return DS_ERR_NULL;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t bytes = (size_t)ctx->n * (size_t)ctx->ld * sizeof(float);
+    cudaError_t e = cudaMemcpyAsync(dev_x, x_host, bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dev_delta, delta_host, bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dev_a, a_host, bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dev_c, c_host, bytes, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+    ds_grad_params gp;
+    gp.a = dev_a; gp.c = dev_c; gp.sigma = sigma; gp.noise = noise;
+    const ds_status st = ds_step(ctx, dev_x, dev_delta, &gp, hp, seed, step, cuda_stream);
+    if (st != DS_OK) return st;
+    e = cudaMemcpyAsync(x_host, dev_x, bytes, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(delta_host, dev_delta, bytes, cudaMemcpyDeviceToHost, stream);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+    return DS_OK;
+}
+
+ds_status ds_noise(float* out, int32_t n, int64_t N, int64_t ld_out, int32_t which, int32_t noise,
+                   uint64_t seed, uint64_t step, void* cuda_stream) {
+    if (!out) return DS_ERR_NULL;
+    if (n < 1 || N < 1 || N >= ((int64_t)1 << 31) || ld_out < N || which < 0 || which > 1 ||
+        noise < DS_NOISE_NONE || noise > DS_NOISE_STUDENT_T3 || step >= ((uint64_t)1 << 56))
+        return DS_ERR_ARG;
+    const cudaError_t e = launch_noise_kernel(out, n, N, ld_out, which, noise, make_rng_step(seed, step),
+                                              static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+    return DS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,76 @@
+// Internal declarations shared by the host API and the kernel translation
+// units of the DeepSqueeze library (not part of the public ABI).
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "ds_device.cuh"
+
+namespace ds {
+
+enum : int { MODE_FUSED = 0, MODE_COMPRESS = 1, MODE_REDUCE = 2 };
+
+// Code formats the kernels are instantiated for.
+enum : int { CODE_SIGN = 0, CODE_U1 = 1, CODE_U2 = 2, CODE_U4 = 3, CODE_U8 = 4, CODE_ID32 = 5 };
+
+struct StepParams {
+    float* x;
+    float* delta;
+    const float* a;
+    const float* c;
+    int64_t ld;
+    int64_t N;
+    int32_t n;
+    int32_t nnz;
+    int64_t tile;             // elements per column tile (= chunk unless prescaled)
+    int64_t tiles;            // column tiles per row
+    const int32_t* row_ptr;   // device CSR of W - I
+    const int32_t* col_idx;
+    const float* wprime;      // W_ij - I_ij, binary32
+    const float* lut;         // reconstruction levels, 2^bits entries
+    uint32_t* codes;
+    int64_t code_pitch;       // words
+    float* scales;
+    int64_t scales_pitch;
+    double* partials;         // [n][tiles], per-node-scale reduction
+    float sigma;
+    float neg_gamma;
+    float eta;
+    RngStep rs;
+    int32_t warps_per_group;  // warps sharing one (node, tile)
+    int32_t nodes_per_block;
+    int32_t prescaled;        // 1: scale of node i is scales[i][0], computed by an earlier launch
+};
+
+struct LaunchShape {
+    int code;                 // CODE_*
+    int noise;                // NOISE_*
+    int elems_per_lane;       // 4, 8 or 16
+    int mode;                 // MODE_*
+    dim3 grid;
+    dim3 block;
+    size_t smem;
+};
+
+// Launchers (defined in the kernel translation units).
+cudaError_t launch_column_fused(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
+cudaError_t launch_column_compress(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
+cudaError_t launch_column_reduce(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
+cudaError_t launch_finalize_scales(const StepParams& p, int code, cudaStream_t stream);
+cudaError_t launch_mix_kernel(const StepParams& p, int code, cudaStream_t stream);
+cudaError_t launch_noise_kernel(float* out, int32_t n, int64_t N, int64_t ld, int which, int noise,
+                                RngStep rs, cudaStream_t stream);
+
+inline int code_bits_of(int code) {
+    switch (code) {
+        case CODE_SIGN: case CODE_U1: return 1;
+        case CODE_U2: return 2;
+        case CODE_U4: return 4;
+        case CODE_U8: return 8;
+        default: return 32;
+    }
+}
+
+}  // namespace ds

@@ -1,0 +1,254 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the
+same seeded inputs.  Packed codes must be bit-exact; x, delta and scales must
+agree within max |gpu - ref| / max |ref| <= 1e-5 per node row after one step
+and 1e-4 after 20 free-running steps."""
+import numpy as np
+import pytest
+
+from paper_1907_07346_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+TOL_STEP = 1e-5
+TOL_RUN = 1e-4
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from oracle import oracle as orc
+    from paper_1907_07346_b200 import binding as B
+    from paper_1907_07346_b200 import build as libbuild
+    libbuild.build()
+    assert torch.cuda.is_available()
+    B.lib()
+    return torch, orc, B
+
+
+def row_rel_err(got, ref):
+    num = np.abs(got.astype(np.float64) - ref.astype(np.float64)).max(axis=1)
+    den = np.maximum(np.abs(ref.astype(np.float64)).max(axis=1), 1e-30)
+    return float((num / den).max())
+
+
+def make_state(graph, N, ld, seed, a_dist="uniform", zero_start=False):
+    rng = np.random.default_rng(seed)
+    n = graph.n
+    a = np.zeros((n, ld), np.float32)
+    c = np.zeros((n, ld), np.float32)
+    x = np.zeros((n, ld), np.float32)
+    d = np.zeros((n, ld), np.float32)
+    if a_dist == "uniform":
+        a[:, :N] = rng.uniform(0.5, 2.0, size=(n, N))
+    else:
+        a[:, :N] = 10.0 ** rng.uniform(-1, 1, size=(n, N))
+    c[:, :N] = rng.standard_normal((n, N))
+    if not zero_start:
+        x[:, :N] = 0.3 * rng.standard_normal((n, N))
+        d[:, :N] = 0.05 * rng.standard_normal((n, N))
+    # padding columns carry sentinels that must survive a step
+    x[:, N:] = 7.0
+    d[:, N:] = -7.0
+    a[:, N:] = 3.0
+    c[:, N:] = 5.0
+    return x, d, a, c
+
+
+def run_case(env, graph, N, kind, bits, chunk, noise, path, steps=1, pad=None, seed=3,
+             sigma=0.1, gamma=0.05, eta=0.5, zero_start=False, tol=TOL_STEP, a_dist="uniform"):
+    torch, orc, B = env
+    ld = I.round_up(N, 4) + (0 if pad is None else pad)
+    x, d, a, c = make_state(graph, N, ld, seed, a_dist, zero_start)
+    ds = B.DeepSqueeze(graph, N, ld, kind, bits, chunk)
+    try:
+        ds.ds_set_path(path)
+    except B.DsError:
+        ds.close()
+        pytest.skip("shape not available on the fused path")
+    assert ds.ds_get_info().path == path
+    dev = [torch.from_numpy(t.copy()).cuda() for t in (x, d, a, c)]
+    worst = 0.0
+    for t in range(steps):
+        codes_ref, scales_ref, _, _ = orc.step(graph, kind, bits, chunk, x, d, a, c, N, sigma, noise,
+                                               gamma, eta, 99 + seed, t)
+        ds.ds_step(dev[0], dev[1], dev[2], dev[3], sigma, noise, gamma, eta, 99 + seed, t)
+        torch.cuda.synchronize()
+        gx, gd = dev[0].cpu().numpy(), dev[1].cpu().numpy()
+        codes, scales = ds.codes_to_host()
+        assert np.array_equal(codes, codes_ref), f"codes differ at step {t}"
+        if scales_ref.shape[1]:
+            assert row_rel_err(scales, scales_ref) <= tol
+        ex, ed = row_rel_err(gx[:, :N], x[:, :N]), row_rel_err(gd[:, :N], d[:, :N])
+        worst = max(worst, ex, ed)
+        assert ex <= tol and ed <= tol, (t, ex, ed)
+        assert np.array_equal(gx[:, N:], x[:, N:]) and np.array_equal(gd[:, N:], d[:, N:])
+    ds.close()
+    return worst
+
+
+# ------------------------------------------------------------ raw streams
+@pytest.mark.parametrize("noise", [I.NOISE_GAUSS, I.NOISE_STUDENT_T3])
+def test_noise_streams_bit_exact(env, noise):
+    torch, orc, B = env
+    n, N = 3, 4099
+    out = torch.zeros((n, 4104), dtype=torch.float32, device="cuda")
+    seed, step = 0xDEADBEEFCAFE, (5 << 32) | 77
+    B.ds_noise(out, n, N, 0, noise, seed, step)
+    got = out.cpu().numpy()
+    for i in range(n):
+        ref = orc.noise_row(noise, seed, i, step, 0, N)
+        assert np.array_equal(got[i, :N].view(np.uint32), ref.view(np.uint32))
+    assert np.all(got[:, N:] == 0)
+
+
+def test_rounding_stream_bit_exact(env):
+    torch, orc, B = env
+    n, N = 2, 1001
+    out = torch.zeros((n, 1004), dtype=torch.float32, device="cuda")
+    B.ds_noise(out, n, N, 1, I.NOISE_NONE, 42, 9)
+    got = out.cpu().numpy()
+    for i in range(n):
+        assert np.array_equal(got[i, :N], orc.rnd24_row(42, i, 9, 0, N))
+
+
+# ---------------------------------------------------------- single steps
+COMPS = [(I.COMP_SIGN1_L1, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 2),
+         (I.COMP_UNIFORM_STOCH_MAXABS, 4), (I.COMP_UNIFORM_STOCH_MAXABS, 8)]
+PATHS = [1, 2]      # DS_PATH_FUSED, DS_PATH_SPLIT
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("comp", COMPS)
+@pytest.mark.parametrize("chunk,N", [(512, 512 * 5 + 1), (256, 256 * 7 + 3), (1024, 1024 * 3 + 130),
+                                     (4096, 4096 * 2 + 74), (32, 32 * 9 + 5), (96, 96 * 4 + 2),
+                                     (512, 200), (512, 512 * 4)])
+def test_single_step_ring(env, path, comp, chunk, N):
+    run_case(env, I.ring(8), N, comp[0], comp[1], chunk, I.NOISE_GAUSS, path)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("gname", ["ring4", "ring16", "torus4x8", "exp64", "exp16"])
+@pytest.mark.parametrize("comp,chunk", [((I.COMP_SIGN1_L1, 1), 1024), ((I.COMP_UNIFORM_STOCH_MAXABS, 4), 512),
+                                        ((I.COMP_UNIFORM_STOCH_MAXABS, 2), 256)])
+def test_single_step_graphs(env, path, gname, comp, chunk):
+    g = {"ring4": I.ring(4), "ring16": I.ring(16), "torus4x8": I.torus(4, 8),
+         "exp64": I.exponential(64), "exp16": I.exponential(16)}[gname]
+    run_case(env, g, chunk * 3 + 41, comp[0], comp[1], chunk, I.NOISE_GAUSS, path)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("noise", [I.NOISE_NONE, I.NOISE_STUDENT_T3])
+def test_single_step_other_noise(env, path, noise):
+    run_case(env, I.torus(4, 8), 256 * 6 + 40, I.COMP_UNIFORM_STOCH_MAXABS, 2, 256, noise, path)
+    run_case(env, I.ring(8), 1024 * 2 + 7, I.COMP_SIGN1_L1, 1, 1024, noise, path)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("comp", [(I.COMP_SIGN1_L1, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 4)])
+@pytest.mark.parametrize("N", [65_536, 1000, 515])
+def test_per_node_scale(env, path, comp, N):
+    run_case(env, I.ring(4), N, comp[0], comp[1], 0, I.NOISE_GAUSS, path)
+
+
+def test_identity_compressor(env):
+    torch, orc, B = env
+    run_case(env, I.ring(8), 1000, I.COMP_IDENTITY, 32, 0, I.NOISE_GAUSS, B.DS_PATH_SPLIT)
+    run_case(env, I.exponential(16), 999, I.COMP_IDENTITY, 32, 64, I.NOISE_NONE, B.DS_PATH_SPLIT)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_padded_pitch(env, path):
+    run_case(env, I.ring(8), 512 * 3 + 2, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_GAUSS, path, pad=28)
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_degenerate_inputs(env, path):
+    """All-zero state and objective: every chunk has scale 0 (b-bit) or 0 (l1)."""
+    torch, orc, B = env
+    g = I.ring(4)
+    N, ld = 700, 704
+    for kind, bits in ((I.COMP_UNIFORM_STOCH_MAXABS, 4), (I.COMP_SIGN1_L1, 1)):
+        ds = B.DeepSqueeze(g, N, ld, kind, bits, 256)
+        ds.ds_set_path(path)
+        z = [np.zeros((4, ld), np.float32) for _ in range(4)]
+        dev = [torch.from_numpy(t.copy()).cuda() for t in z]
+        codes_ref, scales_ref, _, _ = orc.step(g, kind, bits, 256, z[0], z[1], z[2], z[3], N, 0.0,
+                                               I.NOISE_NONE, 0.1, 0.5, 1, 0)
+        ds.ds_step(dev[0], dev[1], dev[2], dev[3], 0.0, I.NOISE_NONE, 0.1, 0.5, 1, 0)
+        torch.cuda.synchronize()
+        codes, scales = ds.codes_to_host()
+        assert np.array_equal(codes, codes_ref) and np.array_equal(scales, scales_ref)
+        assert np.array_equal(dev[0].cpu().numpy(), z[0]) and np.array_equal(dev[1].cpu().numpy(), z[1])
+        ds.close()
+
+
+# ------------------------------------------------- the five workloads, reduced N
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_workloads_free_running_20_steps(env, path, name):
+    """x_0 = delta_0 = 0, 20 free-running steps at a reduced N that still
+    spans several tiles and a ragged tail."""
+    w = I.WORKLOADS[name]
+    N = 65_536 if name == "cfg1" else (w.chunk * 5 + 40)
+    g = w.build_graph()
+    run_case(env, g, N, w.comp_kind, w.bits, w.chunk, w.noise_kind, path, steps=20, seed=5,
+             sigma=w.sigma, gamma=w.gamma, eta=w.eta, zero_start=True, tol=TOL_RUN, a_dist=w.a_dist)
+
+
+def test_same_seed_same_result_and_resume(env):
+    """Counter-based streams: (seed, step) fixes an iteration, so 6 steps equal
+    3 steps, a copy of the state to the host and back, and 3 more."""
+    torch, orc, B = env
+    g = I.ring(8)
+    N, ld = 512 * 4 + 9, 512 * 4 + 12
+    x, d, a, c = make_state(g, N, ld, 1)
+    ds = B.DeepSqueeze(g, N, ld, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512)
+
+    def run(steps, x0, d0, first):
+        dx, dd = torch.from_numpy(x0.copy()).cuda(), torch.from_numpy(d0.copy()).cuda()
+        da, dc = torch.from_numpy(a).cuda(), torch.from_numpy(c).cuda()
+        for t in range(first, first + steps):
+            ds.ds_step(dx, dd, da, dc, 0.1, I.NOISE_GAUSS, 0.02, 0.5, 11, t)
+        torch.cuda.synchronize()
+        return dx.cpu().numpy(), dd.cpu().numpy()
+
+    x6, d6 = run(6, x, d, 0)
+    x3, d3 = run(3, x, d, 0)
+    x33, d33 = run(3, x3, d3, 3)
+    assert np.array_equal(x6, x33) and np.array_equal(d6, d33)
+    ds.close()
+
+
+def test_fused_and_split_paths_agree_bitwise(env):
+    torch, orc, B = env
+    g = I.torus(4, 8)
+    N, ld = 256 * 9 + 40, 256 * 9 + 40
+    x, d, a, c = make_state(g, N, ld, 2)
+    outs = []
+    for path in PATHS:
+        ds = B.DeepSqueeze(g, N, ld, I.COMP_UNIFORM_STOCH_MAXABS, 2, 256)
+        ds.ds_set_path(path)
+        dev = [torch.from_numpy(t.copy()).cuda() for t in (x, d, a, c)]
+        for t in range(3):
+            ds.ds_step(dev[0], dev[1], dev[2], dev[3], 0.1, I.NOISE_STUDENT_T3, 0.005, 0.4, 7, t)
+        torch.cuda.synchronize()
+        outs.append((dev[0].cpu().numpy(), dev[1].cpu().numpy(), *ds.codes_to_host()))
+        ds.close()
+    for u, v in zip(outs[0], outs[1]):
+        assert np.array_equal(u, v)
+
+
+def test_host_buffer_entry_point(env):
+    torch, orc, B = env
+    g = I.ring(8)
+    N, ld = 512 * 3 + 5, 512 * 3 + 8
+    x, d, a, c = make_state(g, N, ld, 4)
+    ds = B.DeepSqueeze(g, N, ld, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512)
+    host = [torch.from_numpy(t.copy()).pin_memory() for t in (x, d, a, c)]
+    dev = [torch.empty((g.n, ld), dtype=torch.float32, device="cuda") for _ in range(4)]
+    ds.ds_step_host(host[0], host[1], host[2], host[3], 0.1, I.NOISE_GAUSS, 0.01, 0.5, 3, 0, *dev)
+    torch.cuda.synchronize()
+    orc.step(g, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, x, d, a, c, N, 0.1, I.NOISE_GAUSS, 0.01, 0.5, 3, 0)
+    assert row_rel_err(host[0].numpy()[:, :N], x[:, :N]) <= TOL_STEP
+    assert row_rel_err(host[1].numpy()[:, :N], d[:, :N]) <= TOL_STEP
+    ds.close()
