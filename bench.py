@@ -1,0 +1,324 @@
+#!/usr/bin/env python
+"""Benchmark of the DeepSqueeze node update on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3]
+    python bench.py --impl reference ...        # times the CPU checker instead
+
+One "step" is one whole iteration of Algorithm 1 for all n nodes (gradient,
+error-compensated compression, residual, gossip mix) on synthetic data of the
+workload's shape.  Metric: node-element updates per second (n * N per step).
+
+With N > 1 GPUs the path does not shard (one GPU simulates all nodes), so every
+rank runs an independent replica of the workload; the reported value is the sum
+of the replicas' updates divided by the slowest rank's time.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_1907_07346_b200 import inputs as I  # noqa: E402
+
+METRIC = "node-element updates/sec per DeepSqueeze step"
+UNIT = "updates/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def algorithmic_bytes_per_update(w: I.Workload) -> float:
+    """Read x, delta, a, c (16 B), write x, delta (8 B), write the codes (b/8 B)
+    and one binary32 scale per chunk (4/chunk B)."""
+    bits = 32 if w.comp_kind == I.COMP_IDENTITY else (1 if w.comp_kind == I.COMP_SIGN1_L1 else w.bits)
+    chunk = w.chunk if w.chunk > 0 else w.N
+    return 24.0 + bits / 8.0 + 4.0 / chunk
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while
+    the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [t.strip() for t in line.split(",")]))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [r for ts, r in self.rows if t0 - 0.05 <= ts <= t1 + 0.15 and len(r) >= 8]
+        if not rows:
+            rows = [r for _, r in self.rows if len(r) >= 8]
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def cpu_baseline(w: I.Workload, a: np.ndarray, c: np.ndarray, sample_cols: int, steps: int = 1,
+                 full_N: int | None = None):
+    """Time the CPU checker, as it stands, on the first `sample_cols` columns
+    of every node of the workload."""
+    from oracle import oracle as orc
+    g = w.build_graph()
+    cols = min(sample_cols, w.N)
+    if w.chunk > 0:
+        cols = max(w.chunk, cols // w.chunk * w.chunk)
+    ld = I.round_up(cols, 4)
+    aa = np.zeros((w.n, ld), np.float32)
+    cc = np.zeros((w.n, ld), np.float32)
+    aa[:, :cols] = a[:, :cols]
+    cc[:, :cols] = c[:, :cols]
+    x = np.zeros((w.n, ld), np.float32)
+    d = np.zeros((w.n, ld), np.float32)
+    times = []
+    for t in range(steps):
+        t0 = time.perf_counter()
+        orc.step(g, w.comp_kind, w.bits, w.chunk, x, d, aa, cc, cols, w.sigma, w.noise_kind,
+                 w.gamma, w.eta, w.seed, t)
+        times.append(time.perf_counter() - t0)
+    return {"value": w.n * cols * steps / sum(times), "unit": UNIT, "cores": orc.num_threads(),
+            "kind": "oracle",
+            "sample": f"{steps} step(s) on the first {cols} of {full_N or w.N} parameters of all {w.n} nodes "
+                      f"({w.n * cols} updates per step)"}, times
+
+
+def run_reference(args, w: I.Workload):
+    """The reference arm: the CPU checker on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = w.with_size(min(w.N, args.ref_cols))
+    a, c = I.objective(sample, I.row_pitch(sample.N))
+    total = args.warmup + args.steps
+    base, times = cpu_baseline(sample, a, c, sample.N, steps=total, full_N=w.N)
+    timed = times[args.warmup:]
+    value = sample.n * min(sample.N, args.ref_cols) * len(timed) / sum(timed)
+    base["value"] = value
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * sum(timed) / len(timed),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "impl": "reference",
+            "config": {"workload": w.describe(), "timed_sample": base["sample"]},
+            "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg3", choices=sorted(I.WORKLOADS))
+    ap.add_argument("--size", type=int, default=0, help="override N (parameters per node)")
+    ap.add_argument("--path", default="auto", choices=["auto", "fused", "split"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-cols", type=int, default=1 << 24,
+                    help="columns per node of the CPU-baseline sample")
+    ap.add_argument("--ref-cols", type=int, default=1 << 21,
+                    help="columns per node of each step of --impl reference")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    w = I.WORKLOADS[args.workload]
+    if args.size:
+        w = w.with_size(args.size)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    from paper_1907_07346_b200 import binding as B
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    g = w.build_graph()
+    ld = I.row_pitch(w.N)
+    a_h, c_h = I.objective(w, ld)
+    ds = B.DeepSqueeze(g, w.N, ld, w.comp_kind, w.bits, w.chunk, device=dev)
+    ds.ds_set_path({"auto": B.DS_PATH_AUTO, "fused": B.DS_PATH_FUSED, "split": B.DS_PATH_SPLIT}[args.path])
+    info = ds.ds_get_info()
+    a = torch.from_numpy(a_h).to(dev)
+    c = torch.from_numpy(c_h).to(dev)
+    x = torch.zeros((w.n, ld), dtype=torch.float32, device=dev)
+    delta = torch.zeros_like(x)
+    stream = torch.cuda.current_stream(dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    step_index = 0
+    for _ in range(args.warmup):
+        ds.ds_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, step_index, stream)
+        step_index += 1
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    t_wall0 = time.time()
+    events[0].record(stream)
+    for k in range(args.steps):
+        ds.ds_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, step_index, stream)
+        step_index += 1
+        events[k + 1].record(stream)
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    total_ms = events[0].elapsed_time(events[-1])
+    per_step = [events[k].elapsed_time(events[k + 1]) for k in range(args.steps)]
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    updates_per_step = w.n * w.N
+    value = world * updates_per_step * args.steps / (total_ms * 1e-3)
+    assert torch.isfinite(x).all() and torch.isfinite(delta).all()
+
+    # Roofline of the dominant kernel.  On the fused path a step IS one launch
+    # of the column kernel, so its average duration is the event time per step.
+    b_alg = algorithmic_bytes_per_update(w)
+    peak, peak_kind = measured_peak()
+    kernel_ms = statistics.mean(per_step)
+    achieved = b_alg * updates_per_step / (kernel_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_source": f"of {peak_kind}",
+                "kernel": "ds_column_kernel (fused)" if info.path == B.DS_PATH_FUSED
+                          else "ds_column_kernel (compress) + ds_mix_kernel",
+                "algorithmic_bytes_per_update": b_alg,
+                "algorithmic_bytes_per_launch": b_alg * updates_per_step,
+                "kernel_ms_mean": kernel_ms, "kernel_ms_min": min(per_step),
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # End to end through the host-buffer entry point: pinned host arrays in,
+    # x and delta back out, every step.
+    e2e = None
+    if not args.no_e2e:
+        hx = torch.zeros((w.n, ld), dtype=torch.float32).pin_memory()
+        hd = torch.zeros((w.n, ld), dtype=torch.float32).pin_memory()
+        ha = torch.from_numpy(a_h).pin_memory()
+        hc = torch.from_numpy(c_h).pin_memory()
+        for t in range(2):
+            ds.ds_step_host(hx, hd, ha, hc, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, t,
+                            x, delta, a, c, stream)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for t in range(args.e2e_steps):
+            ds.ds_step_host(hx, hd, ha, hc, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, 2 + t,
+                            x, delta, a, c, stream)
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        arr_bytes = w.n * ld * 4
+        e2e = {"value": world * updates_per_step * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": 4 * arr_bytes, "d2h_bytes_per_step": 2 * arr_bytes,
+               "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
+               "entry_point": "ds_step_host (pinned host x, delta, a, c in; x, delta out)"}
+        del hx, hd, ha, hc
+
+    base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        base, _ = cpu_baseline(w, a_h, c_h, args.cpu_cols, steps=1)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": w.describe(), "row_pitch": ld,
+                           "path": "fused" if info.path == B.DS_PATH_FUSED else "split",
+                           "elems_per_lane": info.elems_per_lane, "warps_per_chunk": info.warps_per_chunk,
+                           "block_threads": info.block_threads, "grid_blocks": info.grid_blocks,
+                           "l2": "inputs larger than L2 (no flush needed)"
+                                 if 16 * updates_per_step > 4 * 126e6 else "inputs fit in L2: not a roofline point",
+                           "replicas": world},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * info.launches_per_step,
+                "roofline": roofline, "cpu_baseline": base}
+        print(json.dumps(line))
+    ds.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -303,6 +303,10 @@ void oracle_pack_codes(int bits, const uint32_t *q, int64_t first_elem,
  *   scales [n][scales_pitch]    one scale per (node, chunk)
  *   v_out, C_out (optional, [n][N])  the error-compensated variable and its
  *                               decoded compression, for the tests
+ *   k_first                     global index of column 0 in the random streams:
+ *                               0 for a whole problem; a multiple of the chunk
+ *                               length when the arrays hold a window of columns
+ *                               [k_first, k_first + N) of a longer problem
  * Returns 0, or -1 if memory could not be obtained.
  *
  * Operation order per element (one binary32 operation per line):
@@ -325,7 +329,7 @@ int oracle_step(int32_t n, int64_t N, int64_t ld,
                 uint64_t seed, uint64_t step,
                 uint32_t *codes, int64_t code_pitch,
                 float *scales, int64_t scales_pitch,
-                float *v_out, float *C_out)
+                float *v_out, float *C_out, int64_t k_first)
 {
     if (chunk <= 0) chunk = N;
     int code_bits = (comp_kind == COMP_IDENTITY) ? 32
@@ -359,7 +363,7 @@ int oracle_step(int32_t n, int64_t N, int64_t ld,
             for (int64_t kk = 0; kk < m; ++kk) {
                 int64_t k = k0 + kk;
                 size_t at = (size_t)i * (size_t)ld + (size_t)k;
-                float z = oracle_noise_elem(noise_kind, seed, (uint32_t)i, step, k);
+                float z = oracle_noise_elem(noise_kind, seed, (uint32_t)i, step, k_first + k);
                 float d = x[at] - c[at];
                 float nz = sigma * z;
                 float g = fmaf(a[at], d, nz);
@@ -367,7 +371,7 @@ int oracle_step(int32_t n, int64_t N, int64_t ld,
                 h[(size_t)i * (size_t)N + (size_t)k] = hh;
                 v[kk] = hh + delta[at];
                 r[kk] = (comp_kind == COMP_UNIFORM_STOCH_MAXABS)
-                            ? oracle_rnd24_elem(seed, (uint32_t)i, step, k) : 0.0f;
+                            ? oracle_rnd24_elem(seed, (uint32_t)i, step, k_first + k) : 0.0f;
             }
             float s;
             float *Crow = C + (size_t)i * (size_t)N + (size_t)k0;

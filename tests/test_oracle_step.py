@@ -275,3 +275,26 @@ def test_student_t_noise_enters_gradient():
     z = np.stack([orc.noise_row(I.NOISE_STUDENT_T3, 5, i, 2, 0, N) for i in range(4)]).astype(np.float64)
     G = a.astype(np.float64) * (x0.astype(np.float64) - c) + 0.1 * z
     assert np.allclose(v, x0 - 0.05 * G + d0, atol=2e-6, rtol=0)
+
+
+@pytest.mark.parametrize("comp", [(I.COMP_SIGN1_L1, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 4)])
+def test_column_window_equals_slice_of_whole_problem(comp):
+    """Chunks are independent columns: running the iteration on the columns
+    [k_first, k_first + n_cols) alone (random streams indexed by the global
+    column) reproduces that slice of the whole-problem result bit for bit."""
+    g = I.ring(8)
+    chunk, N = 64, 64 * 7 + 10
+    x, d, a, c = make_problem(g, N, 17)
+    xw, dw = x.copy(), d.copy()
+    codes, scales, _, _ = orc.step(g, comp[0], comp[1], chunk, x, d, a, c, N, 0.1, I.NOISE_GAUSS,
+                                   0.05, 0.5, 4, 6)
+    for k_first, n_cols in ((0, 128), (128, 192), (384, N - 384)):
+        sl = slice(k_first, k_first + n_cols)
+        xs, dsl = np.ascontiguousarray(xw[:, sl]), np.ascontiguousarray(dw[:, sl])
+        cw, sw, _, _ = orc.step(g, comp[0], comp[1], chunk, xs, dsl,
+                                np.ascontiguousarray(a[:, sl]), np.ascontiguousarray(c[:, sl]),
+                                n_cols, 0.1, I.NOISE_GAUSS, 0.05, 0.5, 4, 6, k_first=k_first)
+        assert np.array_equal(xs, x[:, sl]) and np.array_equal(dsl, d[:, sl])
+        assert np.array_equal(sw, scales[:, k_first // chunk:k_first // chunk + sw.shape[1]])
+        w0 = k_first * comp[1] // 32
+        assert np.array_equal(cw, codes[:, w0:w0 + cw.shape[1]])
