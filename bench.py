@@ -169,7 +169,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg3", choices=sorted(I.WORKLOADS))
     ap.add_argument("--size", type=int, default=0, help="override N (parameters per node)")
-    ap.add_argument("--path", default="auto", choices=["auto", "fused", "split"])
+    ap.add_argument("--path", default="auto", choices=["auto", "fused", "fused_ldg", "split"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-cols", type=int, default=1 << 24,
@@ -208,7 +208,8 @@ def main():
     ld = I.row_pitch(w.N)
     a_h, c_h = I.objective(w, ld)
     ds = B.DeepSqueeze(g, w.N, ld, w.comp_kind, w.bits, w.chunk, device=dev)
-    ds.ds_set_path({"auto": B.DS_PATH_AUTO, "fused": B.DS_PATH_FUSED, "split": B.DS_PATH_SPLIT}[args.path])
+    ds.ds_set_path({"auto": B.DS_PATH_AUTO, "fused": B.DS_PATH_FUSED, "fused_ldg": B.DS_PATH_FUSED_LDG,
+                    "split": B.DS_PATH_SPLIT}[args.path])
     info = ds.ds_get_info()
     a = torch.from_numpy(a_h).to(dev)
     c = torch.from_numpy(c_h).to(dev)
@@ -249,6 +250,7 @@ def main():
         total_ms = float(t.item())
     updates_per_step = w.n * w.N
     value = world * updates_per_step * args.steps / (total_ms * 1e-3)
+    ds.ds_sync(stream)
     assert torch.isfinite(x).all() and torch.isfinite(delta).all()
 
     # Roofline of the dominant kernel.  On the fused path a step IS one launch
@@ -259,8 +261,8 @@ def main():
     achieved = b_alg * updates_per_step / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": None, "peak_source": f"of {peak_kind}",
-                "kernel": "ds_column_kernel (fused)" if info.path == B.DS_PATH_FUSED
-                          else "ds_column_kernel (compress) + ds_mix_kernel",
+                "kernel": {B.DS_PATH_FUSED: "ds_fused_tma_kernel", B.DS_PATH_FUSED_LDG: "ds_column_kernel (fused)",
+                           B.DS_PATH_SPLIT: "ds_column_kernel (compress) + ds_mix_kernel"}[info.path],
                 "algorithmic_bytes_per_update": b_alg,
                 "algorithmic_bytes_per_launch": b_alg * updates_per_step,
                 "kernel_ms_mean": kernel_ms, "kernel_ms_min": min(per_step),
@@ -306,7 +308,8 @@ def main():
                 "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": w.describe(), "row_pitch": ld,
-                           "path": "fused" if info.path == B.DS_PATH_FUSED else "split",
+                           "path": {B.DS_PATH_FUSED: "fused (persistent, TMA-staged)",
+                                    B.DS_PATH_FUSED_LDG: "fused (direct loads)", B.DS_PATH_SPLIT: "split"}[info.path],
                            "elems_per_lane": info.elems_per_lane, "warps_per_chunk": info.warps_per_chunk,
                            "block_threads": info.block_threads, "grid_blocks": info.grid_blocks,
                            "l2": "inputs larger than L2 (no flush needed)"

@@ -50,7 +50,8 @@ typedef enum {
     DS_ERR_ALIGN = 7,            /* pointer not 16-byte aligned, or pitch not a multiple of 4 */
     DS_ERR_WORKSPACE = 8,        /* workspace smaller than ds_workspace_size() */
     DS_ERR_UNSUPPORTED = 9,      /* combination not implemented (e.g. bits not in {1,2,4,8}) */
-    DS_ERR_CUDA = 10             /* a CUDA runtime call failed (no device, launch error, ...) */
+    DS_ERR_CUDA = 10,            /* a CUDA runtime call failed (no device, launch error, ...) */
+    DS_ERR_TIMEOUT = 11          /* a bounded wait inside a kernel ran out; x, delta are incomplete */
 } ds_status;
 
 /* Node graph in CSR form, HOST memory: row i lists N(i) in ascending order
@@ -105,13 +106,19 @@ typedef struct {
 } ds_hparams;
 
 /* How a step is executed.
- *   DS_PATH_FUSED  one kernel: a thread block owns one chunk column of ALL nodes, keeps
- *                  x - gamma g in registers and the column's codes in shared memory, and
- *                  mixes without re-reading anything from global memory.
- *   DS_PATH_SPLIT  two kernels: compress (x - gamma g written into x, codes to the
- *                  workspace), then mix (codes re-read).  Works for every shape.
- *   DS_PATH_AUTO   fused when the shape allows it, else split. */
-typedef enum { DS_PATH_AUTO = 0, DS_PATH_FUSED = 1, DS_PATH_SPLIT = 2 } ds_path;
+ *   DS_PATH_FUSED      one kernel: a thread block owns one chunk column of ALL nodes, keeps
+ *                      x - gamma g in registers and the column's C[v] in shared memory, and
+ *                      mixes without re-reading anything from global memory.  Where the
+ *                      column fits in shared memory this is the persistent kernel whose
+ *                      inputs are staged by bulk asynchronous copies (TMA); otherwise the
+ *                      variant below.
+ *   DS_PATH_FUSED_LDG  the fused kernel with direct vector loads and packed codes in shared
+ *                      memory (one block per column).
+ *   DS_PATH_SPLIT      two kernels: compress (x - gamma g written into x, codes to the
+ *                      workspace), then mix (each neighbour's packed codes streamed once and
+ *                      decoded in registers).  Works for every shape.
+ *   DS_PATH_AUTO       the first of the three that the shape allows. */
+typedef enum { DS_PATH_AUTO = 0, DS_PATH_FUSED = 1, DS_PATH_SPLIT = 2, DS_PATH_FUSED_LDG = 3 } ds_path;
 
 typedef struct {
     int32_t path;               /* ds_path actually used by ds_step */
@@ -180,6 +187,12 @@ ds_status ds_set_path(ds_ctx *ctx, int32_t path);
 
 /* Launch geometry of the current path (host-only). */
 ds_status ds_get_info(const ds_ctx *ctx, ds_info *info);
+
+/* Wait for the stream and report whether any kernel of this context gave up on
+ * a bounded wait since the last call (DS_ERR_TIMEOUT; the flag is cleared).
+ * The kernels never spin without a limit: a copy that does not arrive ends
+ * the step early instead of hanging the device. */
+ds_status ds_sync(ds_ctx *ctx, void *cuda_stream);
 
 /* Diagnostics: write the random streams the kernels draw from, one value per
  * element, out[node][k] for k < N (device, [n][ld_out]).  which = 0: unit

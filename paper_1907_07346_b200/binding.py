@@ -16,14 +16,15 @@ LIB_PATH = os.path.join(_HERE, "libdeepsqueeze.so")
 
 DS_OK = 0
 (DS_ERR_NULL, DS_ERR_ARG, DS_ERR_GRAPH, DS_ERR_W_NOT_SYMMETRIC, DS_ERR_W_NOT_STOCHASTIC,
- DS_ERR_NO_SELF_LOOP, DS_ERR_ALIGN, DS_ERR_WORKSPACE, DS_ERR_UNSUPPORTED, DS_ERR_CUDA) = range(1, 11)
+ DS_ERR_NO_SELF_LOOP, DS_ERR_ALIGN, DS_ERR_WORKSPACE, DS_ERR_UNSUPPORTED, DS_ERR_CUDA,
+ DS_ERR_TIMEOUT) = range(1, 12)
 
 DS_COMP_IDENTITY, DS_COMP_SIGN1_L1, DS_COMP_UNIFORM_STOCH_MAXABS = 0, 1, 2
 DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
-DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT = 0, 1, 2
+DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 
 EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_host", "ds_codes", "ds_set_path",
-           "ds_get_info", "ds_noise", "ds_destroy", "ds_strerror"]
+           "ds_get_info", "ds_sync", "ds_noise", "ds_destroy", "ds_strerror"]
 
 
 class ds_graph(C.Structure):
@@ -77,6 +78,8 @@ def lib():
         L.ds_set_path.restype = C.c_int
         L.ds_get_info.argtypes = [C.c_void_p, C.POINTER(ds_info)]
         L.ds_get_info.restype = C.c_int
+        L.ds_sync.argtypes = [C.c_void_p, C.c_void_p]
+        L.ds_sync.restype = C.c_int
         L.ds_noise.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
                                C.c_uint64, C.c_uint64, C.c_void_p]
         L.ds_noise.restype = C.c_int
@@ -178,6 +181,11 @@ class DeepSqueeze:
                                   c_h.data_ptr(), sigma, noise, C.byref(hp), seed, step,
                                   dev_x.data_ptr(), dev_delta.data_ptr(), dev_a.data_ptr(),
                                   dev_c.data_ptr(), C.c_void_p(s.cuda_stream)), "ds_step_host")
+
+    def ds_sync(self, stream=None):
+        """Synchronise the stream and raise if a kernel gave up on a bounded wait."""
+        s = self.torch.cuda.current_stream(self.device) if stream is None else stream
+        _check(lib().ds_sync(self.ctx, C.c_void_p(s.cuda_stream)), "ds_sync")
 
     def ds_codes(self):
         """(codes_ptr, code_pitch_words, scales_ptr, scales_pitch) of the last step."""

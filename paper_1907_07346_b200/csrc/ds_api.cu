@@ -7,7 +7,7 @@
 #include <vector>
 
 #include "../../include/deepsqueeze.h"
-#include "ds_column_kernel.cuh"
+#include "ds_fused_tma_kernel.cuh"
 
 using namespace ds;
 
@@ -32,7 +32,7 @@ struct Shape {
 };
 
 struct WsLayout {
-    size_t codes, scales, partials, row_ptr, col_idx, wprime, lut, total;
+    size_t codes, scales, partials, row_ptr, col_idx, wprime, lut, error_flag, total;
 };
 
 bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
@@ -76,6 +76,7 @@ WsLayout make_ws(int32_t n, int32_t nnz, const Shape& sh) {
     w.col_idx = off;  off = align_up(off + (size_t)nnz * 4, kAlign);
     w.wprime = off;   off = align_up(off + (size_t)nnz * 4, kAlign);
     w.lut = off;      off = align_up(off + 256 * 4, kAlign);
+    w.error_flag = off; off = align_up(off + 4, kAlign);
     w.total = off;
     return w;
 }
@@ -120,6 +121,25 @@ Plan plan_column(int mode, const Shape& sh, int32_t n, int32_t nnz) {
     return pl;
 }
 
+Plan plan_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms) {
+    Plan pl;
+    int E, G;
+    pick_lane_shape(sh.tile, &E, &G);
+    pl.elems_per_lane = E;
+    pl.warps_per_group = G;
+    if (sh.code == CODE_ID32 || (int64_t)n * G > 32 || num_sms < 1) return pl;
+    // every warp of a group owns a whole E*32-element segment
+    if ((int64_t)G * E * 32 < sh.tile) return pl;
+    pl.nodes_per_block = n;
+    pl.block = dim3((unsigned)(n * G * 32));
+    const bool lut = (sh.code != CODE_SIGN);
+    pl.smem = tma_smem_layout(lut, E, n * G, G, sh.tile, n, nnz).total;
+    if (pl.smem > (size_t)kMaxSmem) return pl;
+    pl.grid = dim3((unsigned)std::min<int64_t>(sh.tiles, num_sms));
+    pl.ok = true;
+    return pl;
+}
+
 }  // namespace
 
 struct ds_ctx {
@@ -130,7 +150,8 @@ struct ds_ctx {
     WsLayout ws;
     unsigned char* base;
     int path_req;
-    Plan fused, compress, reduce;
+    Plan tma, fused, compress, reduce;
+    int num_sms;
 };
 
 extern "C" {
@@ -148,6 +169,7 @@ const char* ds_strerror(ds_status status) {
         case DS_ERR_WORKSPACE: return "workspace too small";
         case DS_ERR_UNSUPPORTED: return "unsupported combination";
         case DS_ERR_CUDA: return "CUDA runtime error";
+        case DS_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out; the step is incomplete";
     }
     return "unknown status";
 }
@@ -221,10 +243,19 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     ctx->comp = *comp; ctx->sh = sh; ctx->ws = ws;
     ctx->base = static_cast<unsigned char*>(workspace);
     ctx->path_req = DS_PATH_AUTO;
-    ctx->fused = plan_column(MODE_FUSED, sh, n, nnz);
     ctx->compress = plan_column(MODE_COMPRESS, sh, n, nnz);
     ctx->reduce = plan_column(MODE_REDUCE, sh, n, nnz);
     if (!ctx->compress.ok) { delete ctx; return DS_ERR_UNSUPPORTED; }
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        (void)cudaGetLastError();
+        delete ctx;
+        return DS_ERR_CUDA;
+    }
+    ctx->num_sms = sms;
+    ctx->tma = plan_tma(sh, n, nnz, sms);
+    ctx->fused = plan_column(MODE_FUSED, sh, n, nnz);
 
     // w'_ij = W_ij - I_ij in binary32; reconstruction levels (2q - L)/L.
     std::vector<float> wprime((size_t)nnz);
@@ -243,6 +274,7 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.lut, lut, sizeof(lut), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.codes, 0, ws.scales - ws.codes);
     if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.scales, 0, ws.partials - ws.scales);
+    if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.error_flag, 0, 4);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         delete ctx;
@@ -254,24 +286,29 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
 
 void ds_destroy(ds_ctx* ctx) { delete ctx; }
 
-static bool use_fused(const ds_ctx* ctx) {
-    if (ctx->path_req == DS_PATH_SPLIT) return false;
-    return ctx->fused.ok;
+// 2: persistent TMA-staged fused kernel, 1: fused kernel with direct loads, 0: two kernels
+static int fused_kind(const ds_ctx* ctx) {
+    if (ctx->path_req == DS_PATH_SPLIT) return 0;
+    if (ctx->path_req == DS_PATH_FUSED_LDG) return ctx->fused.ok ? 1 : 0;
+    if (ctx->tma.ok) return 2;
+    return ctx->fused.ok ? 1 : 0;
 }
 
 ds_status ds_set_path(ds_ctx* ctx, int32_t path) {
     if (!ctx) return DS_ERR_NULL;
-    if (path < DS_PATH_AUTO || path > DS_PATH_SPLIT) return DS_ERR_ARG;
-    if (path == DS_PATH_FUSED && !ctx->fused.ok) return DS_ERR_UNSUPPORTED;
+    if (path < DS_PATH_AUTO || path > DS_PATH_FUSED_LDG) return DS_ERR_ARG;
+    if (path == DS_PATH_FUSED && !ctx->fused.ok && !ctx->tma.ok) return DS_ERR_UNSUPPORTED;
+    if (path == DS_PATH_FUSED_LDG && !ctx->fused.ok) return DS_ERR_UNSUPPORTED;
     ctx->path_req = path;
     return DS_OK;
 }
 
 ds_status ds_get_info(const ds_ctx* ctx, ds_info* info) {
     if (!ctx || !info) return DS_ERR_NULL;
-    const bool fused = use_fused(ctx);
-    const Plan& pl = fused ? ctx->fused : ctx->compress;
-    info->path = fused ? DS_PATH_FUSED : DS_PATH_SPLIT;
+    const int kind = fused_kind(ctx);
+    const bool fused = kind != 0;
+    const Plan& pl = (kind == 2) ? ctx->tma : (kind == 1) ? ctx->fused : ctx->compress;
+    info->path = (kind == 2) ? DS_PATH_FUSED : (kind == 1) ? DS_PATH_FUSED_LDG : DS_PATH_SPLIT;
     info->launches_per_step = (fused ? 1 : 2) + (ctx->sh.per_node ? 2 : 0);
     info->elems_per_lane = pl.elems_per_lane;
     info->warps_per_chunk = pl.warps_per_group;
@@ -315,6 +352,7 @@ ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp,
     p.scales = reinterpret_cast<float*>(ctx->base + ctx->ws.scales);
     p.scales_pitch = ctx->sh.scales_pitch;
     p.partials = reinterpret_cast<double*>(ctx->base + ctx->ws.partials);
+    p.error_flag = reinterpret_cast<int*>(ctx->base + ctx->ws.error_flag);
     p.sigma = gp->sigma;
     p.neg_gamma = -hp->gamma;
     p.eta = hp->eta;
@@ -335,7 +373,12 @@ ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp,
         if (e == cudaSuccess) e = launch_finalize_scales(p, ctx->sh.code, stream);
     }
     if (e == cudaSuccess) {
-        if (use_fused(ctx)) {
+        const int kind = fused_kind(ctx);
+        if (kind == 2) {
+            p.warps_per_group = ctx->tma.warps_per_group;
+            p.nodes_per_block = ctx->tma.nodes_per_block;
+            e = launch_fused_tma(shape_of(ctx->tma, MODE_FUSED), p, stream);
+        } else if (kind == 1) {
             p.warps_per_group = ctx->fused.warps_per_group;
             p.nodes_per_block = ctx->fused.nodes_per_block;
             e = launch_column_fused(shape_of(ctx->fused, MODE_FUSED), p, stream);
@@ -374,6 +417,19 @@ ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const floa
     e = cudaMemcpyAsync(x_host, dev_x, bytes, cudaMemcpyDeviceToHost, stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(delta_host, dev_delta, bytes, cudaMemcpyDeviceToHost, stream);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+    return DS_OK;
+}
+
+ds_status ds_sync(ds_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return DS_ERR_NULL;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+    int flag = 0;
+    if (e == cudaSuccess) e = cudaMemcpy(&flag, ctx->base + ctx->ws.error_flag, 4, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+    if (flag != 0) {
+        (void)cudaMemset(ctx->base + ctx->ws.error_flag, 0, 4);
+        return DS_ERR_TIMEOUT;
+    }
     return DS_OK;
 }
 

@@ -26,7 +26,7 @@
 namespace ds {
 
 struct SmemLayout {
-    uint32_t codes_off, scale_off, red_off, lut_off, rowptr_off, col_off, w_off, total;
+    uint32_t codes_off, scale_off, table_off, red_off, lut_off, rowptr_off, col_off, w_off, total;
     uint32_t cw;   // code words per (node, tile)
 };
 
@@ -41,6 +41,9 @@ __host__ __device__ inline SmemLayout smem_layout(int mode, int code_bits, bool 
     off += (mode == MODE_FUSED) ? 2u * (uint32_t)npb * L.cw * 4u : 0u;
     L.scale_off = off;
     off += (mode == MODE_FUSED) ? 2u * (uint32_t)npb * 4u : 0u;
+    // decode tables s_j * level[q] of the tile, for codes of up to 4 bits
+    L.table_off = off;
+    off += (mode == MODE_FUSED && has_lut && code_bits <= 4) ? 2u * (uint32_t)npb * 16u * 4u : 0u;
     L.lut_off = off;
     off += has_lut ? 256u * 4u : 0u;
     L.rowptr_off = off;
@@ -62,6 +65,7 @@ struct CodeTraits {
                                : (CODE == CODE_U4) ? 4
                                : (CODE == CODE_U8) ? 8 : 32;
     static constexpr bool kLut = !(kSign || kIdentity);
+    static constexpr bool kTable = kLut && kBits <= 4;   // per-node decode table in shared memory
     // lanes whose four-element pieces share one 32-bit code word
     static constexpr int kLanesPerWord = (kBits >= 8) ? 1 : 8 / kBits;
     static constexpr uint32_t kPieceMask = (kBits >= 8) ? 0xffffffffu : ((1u << (4 * kBits)) - 1u);
@@ -169,6 +173,10 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
     }
     if constexpr (MODE == MODE_REDUCE) return;
     const bool degenerate = (!T::kSign && !T::kIdentity && s == 0.0f);
+    // the quotient v/s may use the reciprocal only while s is far from the
+    // ends of the exponent range (uniform over the group)
+    const bool fast = T::kLut && s >= 0x1p-60f && s <= 0x1p+60f;
+    const float inv_s = fast ? __fdiv_rn(1.0f, s) : 0.0f;
 
     const float* lut = reinterpret_cast<const float*>(smem + L.lut_off);
     uint32_t* codes_sm = reinterpret_cast<uint32_t*>(smem + L.codes_off) + (size_t)buf * p.nodes_per_block * L.cw;
@@ -205,12 +213,22 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
                         dn[j] = __fadd_rn(v[4 * r + j], -cv);
                         if (FULL || j < nv) piece |= bit << j;
                     }
+                } else if (fast) {
+                    const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node, (uint32_t)(k0 + e0));
+                    const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t q = quantise_recip(v[4 * r + j], s, inv_s, rv[j], kHalfL, (int)kL);
+                        const float cv = __fmul_rn(s, lut[q]);
+                        dn[j] = __fadd_rn(v[4 * r + j], -cv);
+                        if (FULL || j < nv) piece |= q << (T::kBits * j);
+                    }
                 } else {
                     const float4 rr = rnd24x4(p.rs, (uint32_t)node, (uint32_t)(k0 + e0));
                     const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint32_t q = degenerate ? 0u : quantise(v[4 * r + j], s, rv[j], kHalfL, kL);
+                        const uint32_t q = degenerate ? 0u : quantise(v[4 * r + j], s, rv[j], kHalfL, (int)kL);
                         const float cv = __fmul_rn(s, lut[q]);
                         dn[j] = __fadd_rn(v[4 * r + j], -cv);
                         if (FULL || j < nv) piece |= q << (T::kBits * j);
@@ -241,6 +259,10 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
 
     if constexpr (MODE == MODE_FUSED) {
         if (wg == 0 && lane == 0) scale_sm[grp] = s;
+        float* table_sm = reinterpret_cast<float*>(smem + L.table_off) + buf * p.nodes_per_block * 16;
+        if constexpr (T::kTable) {
+            if (wg == 0 && lane < (1 << T::kBits)) table_sm[grp * 16 + lane] = __fmul_rn(s, lut[lane]);
+        }
         __syncthreads();    // codes and scales of all nodes of this tile are in shared memory
 
         // the tile's packed codes leave for global memory ("send")
@@ -260,6 +282,7 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
             const int j = cj[e];
             const float w = wp[e];
             const float sj = scale_sm[j];
+            const float* table_j = table_sm + j * 16;
             const uint32_t* row_j = codes_sm + (size_t)j * L.cw;
 #pragma unroll
             for (int r = 0; r < V; ++r) {
@@ -275,7 +298,8 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
                         cv = __uint_as_float(__float_as_uint(sj) ^ neg);
                     } else {
                         const uint32_t q = (piece >> (T::kBits * t)) & ((1u << T::kBits) - 1u);
-                        cv = __fmul_rn(sj, lut[q]);
+                        if constexpr (T::kTable) cv = table_j[q];
+                        else cv = __fmul_rn(sj, lut[q]);
                     }
                     acc[4 * r + t] = __fmaf_rn(w, cv, acc[4 * r + t]);
                 }

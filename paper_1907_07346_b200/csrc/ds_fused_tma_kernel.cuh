@@ -1,0 +1,353 @@
+// Persistent fused kernel with TMA-staged inputs (sm_100a).
+//
+// One thread block per SM walks over the column tiles.  A group of G warps
+// owns one (node, tile); every warp owns a contiguous segment of E*32 elements
+// of it and a private shared-memory slot holding that segment of x, delta, a
+// and c.  The slot is filled by four bulk asynchronous copies
+// (cp.async.bulk global -> shared, completion counted on the warp's own
+// mbarrier) that the warp issues for its NEXT tile as soon as it has moved the
+// current tile into registers, so the copy of tile t+1 runs under the
+// compression and mixing of tile t and no warp waits for DRAM in steady state.
+//
+// The decoded compression C[v] of the tile is kept in shared memory as
+// binary32 (double buffered): the node that produced it has it in registers
+// anyway, and each neighbour reads it back with 128-bit shared loads, so the
+// local update of Algorithm 1 costs one fma per (element, neighbour).  The
+// packed codes and the scales still go to global memory: they are what the
+// node "sends".
+//
+// Every wait on an mbarrier is bounded.  A warp whose copy does not arrive
+// gives up, raises the step's error flag and drops out of the tile without
+// storing; the block leaves the tile loop together at the next barrier.
+#pragma once
+
+#include "ds_column_kernel.cuh"
+
+namespace ds {
+
+struct TmaSmemLayout {
+    uint32_t slots_off, cval_off, red_off, lut_off, rowptr_off, col_off, w_off, mbar_off, abort_off, total;
+    uint32_t seg_bytes;    // bytes of one array segment of one warp
+};
+
+__host__ __device__ inline TmaSmemLayout tma_smem_layout(bool has_lut, int E, int nwarps, int G,
+                                                         int64_t tile, int n, int nnz) {
+    TmaSmemLayout L;
+    uint32_t off = 0;
+    L.seg_bytes = (uint32_t)E * 32u * 4u;
+    L.slots_off = off;   off += (uint32_t)nwarps * 4u * L.seg_bytes;
+    L.cval_off = off;    off += 2u * (uint32_t)n * (uint32_t)tile * 4u;
+    L.red_off = off;     off += (G > 1) ? (uint32_t)nwarps * 8u : 0u;
+    L.mbar_off = off;    off += (uint32_t)nwarps * 8u;
+    L.lut_off = off;     off += has_lut ? 256u * 4u : 0u;
+    L.rowptr_off = off;  off += (uint32_t)(n + 1) * 4u;
+    L.col_off = off;     off += (uint32_t)nnz * 4u;
+    L.w_off = off;       off += (uint32_t)nnz * 4u;
+    L.abort_off = off;   off += 8u;
+    L.total = (off + 127u) & ~127u;
+    return L;
+}
+
+// ---- thin wrappers over the PTX of mbarriers and bulk copies ----------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0u;
+}
+// Bounded wait: false if the phase did not complete within the try budget.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t tries = 0; tries < (1u << 22); ++tries)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+template <int CODE, int NOISE, int E, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_constant__ StepParams p) {
+    using T = CodeTraits<CODE>;
+    static_assert(!T::kIdentity, "the identity compressor runs on the two-kernel path");
+    constexpr int V = E / 4;
+    constexpr int SEG = E * 32;                       // elements per warp segment
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int G = p.warps_per_group;
+    const int nwarps = blockDim.x >> 5;
+    const TmaSmemLayout L = tma_smem_layout(T::kLut, E, nwarps, G, p.tile, p.n, p.nnz);
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int node = warp / G;                        // the block holds all n nodes
+    const int wg = warp - node * G;
+    const int seg0 = wg * SEG;                        // first element of this warp's segment in the tile
+
+    float* lut = reinterpret_cast<float*>(smem + L.lut_off);
+    int32_t* rp = reinterpret_cast<int32_t*>(smem + L.rowptr_off);
+    int32_t* cj = reinterpret_cast<int32_t*>(smem + L.col_off);
+    float* wp = reinterpret_cast<float*>(smem + L.w_off);
+    volatile int* abort_sm = reinterpret_cast<volatile int*>(smem + L.abort_off);
+    const float* slot = reinterpret_cast<const float*>(smem + L.slots_off + (size_t)warp * 4u * L.seg_bytes);
+    const uint32_t slot_addr = smem_u32(slot);
+    const uint32_t bar = smem_u32(smem + L.mbar_off + warp * 8);
+
+    if constexpr (T::kLut)
+        for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x) lut[t] = p.lut[t];
+    for (int t = threadIdx.x; t <= p.n; t += blockDim.x) rp[t] = p.row_ptr[t];
+    for (int t = threadIdx.x; t < p.nnz; t += blockDim.x) { cj[t] = p.col_idx[t]; wp[t] = p.wprime[t]; }
+    if (threadIdx.x < 2) abort_sm[threadIdx.x] = 0;
+    if (lane == 0) mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+
+    // Valid elements of this warp's segment in tile `col`, and the copy that fetches them.
+    auto seg_len_of = [&](int64_t col) -> int {
+        const int64_t remain = p.N - col * p.tile;
+        const int m_len = (int)(remain < p.tile ? remain : p.tile);
+        return min(max(m_len - seg0, 0), SEG);
+    };
+    auto issue = [&](int64_t col) -> bool {
+        const int len = seg_len_of(col);
+        if (len <= 0) return false;
+        if (lane == 0) {
+            const uint32_t bytes = (uint32_t)((len + 3) & ~3) * 4u;
+            const size_t at = (size_t)node * (size_t)p.ld + (size_t)(col * p.tile) + (size_t)seg0;
+            fence_proxy_async();      // earlier generic reads of the slot are ordered before the refill
+            mbar_expect_tx(bar, 4u * bytes);
+            bulk_g2s(slot_addr + 0u * L.seg_bytes, p.x + at, bytes, bar);
+            bulk_g2s(slot_addr + 1u * L.seg_bytes, p.delta + at, bytes, bar);
+            bulk_g2s(slot_addr + 2u * L.seg_bytes, p.a + at, bytes, bar);
+            bulk_g2s(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar);
+        }
+        return true;
+    };
+
+    int64_t col = blockIdx.x;
+    bool pending = (col < p.tiles) ? issue(col) : false;
+    uint32_t parity = 0;
+    int buf = 0;
+    constexpr float kL = (float)((1u << (T::kBits & 15)) - 1u);
+    constexpr float kHalfL = 0.5f * kL;
+
+    for (; col < p.tiles; col += gridDim.x) {
+        const int64_t k0 = col * p.tile;
+        const int64_t remain = p.N - k0;
+        const int m_len = (int)(remain < p.tile ? remain : p.tile);
+        const int seg_len = min(max(m_len - seg0, 0), SEG);
+        const size_t row = (size_t)node * (size_t)p.ld + (size_t)k0 + (size_t)seg0;
+        float* cval = reinterpret_cast<float*>(smem + L.cval_off) + (size_t)buf * p.n * p.tile;
+
+        // ---- wait for this tile's segment --------------------------------
+        bool alive = true;
+        if (pending) {
+            alive = mbar_wait_bounded(bar, parity);
+            parity ^= 1u;
+            if (!alive) {
+                abort_sm[buf] = 1;
+                if (lane == 0) *p.error_flag = 1;
+            }
+        }
+        const int live_len = alive ? seg_len : 0;
+        const bool full = (live_len == SEG);
+
+        // ---- phase A: slot -> registers, local step, scale partial ---------
+        float h[E], v[E];
+        double sum = 0.0;
+        float mx = 0.0f;
+#pragma unroll
+        for (int r = 0; r < V; ++r) {
+            const int e0 = 4 * (32 * r + lane);              // offset inside the segment
+            const int nv = full ? 4 : min(max(live_len - e0, 0), 4);
+            if (nv > 0) {
+                const float4 x4 = *reinterpret_cast<const float4*>(slot + 0 * SEG + e0);
+                const float4 d4 = *reinterpret_cast<const float4*>(slot + 1 * SEG + e0);
+                const float4 a4 = *reinterpret_cast<const float4*>(slot + 2 * SEG + e0);
+                const float4 c4 = *reinterpret_cast<const float4*>(slot + 3 * SEG + e0);
+                const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                local_step(x4.x, d4.x, a4.x, c4.x, z4.x, p.sigma, p.neg_gamma, h[4 * r + 0], v[4 * r + 0]);
+                local_step(x4.y, d4.y, a4.y, c4.y, z4.y, p.sigma, p.neg_gamma, h[4 * r + 1], v[4 * r + 1]);
+                local_step(x4.z, d4.z, a4.z, c4.z, z4.z, p.sigma, p.neg_gamma, h[4 * r + 2], v[4 * r + 2]);
+                local_step(x4.w, d4.w, a4.w, c4.w, z4.w, p.sigma, p.neg_gamma, h[4 * r + 3], v[4 * r + 3]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
+                    if constexpr (T::kSign) sum += (double)fabsf(v[4 * r + j]);
+                    else mx = fmaxf(mx, fabsf(v[4 * r + j]));
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
+            }
+        }
+        // the slot is in registers: refill it with the segment of the next tile
+        __syncwarp();
+        {
+            const int64_t next = col + gridDim.x;
+            pending = (next < p.tiles) ? issue(next) : false;
+        }
+
+        // ---- scale of the (node, tile) -----------------------------------
+        float s;
+        if (p.prescaled) {
+            s = p.scales[(size_t)node * (size_t)p.scales_pitch];
+        } else {
+            double part;
+            if constexpr (T::kSign) part = warp_sum(sum);
+            else part = (double)__uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
+            if (G > 1) {
+                double* red = reinterpret_cast<double*>(smem + L.red_off);
+                if (lane == 0) red[warp] = part;
+                __syncthreads();
+                part = 0.0;
+                for (int w = 0; w < G; ++w) {
+                    const double t = red[node * G + w];
+                    if constexpr (T::kSign) part += t;
+                    else part = fmax(part, t);
+                }
+            }
+            if constexpr (T::kSign) {
+                s = (float)(part / (double)m_len);
+            } else {
+                s = (float)part;
+                if (s == 0.0f || !(fabsf(s) <= 3.402823466e+38f)) s = 0.0f;
+            }
+        }
+        const bool degenerate = (!T::kSign && s == 0.0f);
+        const bool fast = T::kLut && s >= 0x1p-60f && s <= 0x1p+60f;
+        const float inv_s = fast ? __fdiv_rn(1.0f, s) : 0.0f;
+        const size_t code_row = (size_t)node * (size_t)p.code_pitch + (size_t)(((k0 + seg0) * T::kBits) >> 5);
+        float* cval_mine = cval + (size_t)node * p.tile + seg0;
+
+        // ---- phase B: compress, residual, pack -----------------------------
+#pragma unroll
+        for (int r = 0; r < V; ++r) {
+            const int f = 32 * r + lane;                     // float4 index inside the segment
+            const int e0 = 4 * f;
+            const int nv = full ? 4 : min(max(live_len - e0, 0), 4);
+            uint32_t piece = 0u;
+            if (nv > 0) {
+                float dn[4], cv[4];
+                if constexpr (T::kSign) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t bit = (v[4 * r + j] >= 0.0f) ? 1u : 0u;
+                        cv[j] = bit ? s : -s;
+                        if (j < nv) piece |= bit << j;
+                    }
+                } else if (fast) {
+                    const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                    const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t q = quantise_recip(v[4 * r + j], s, inv_s, rv[j], kHalfL, (int)kL);
+                        cv[j] = __fmul_rn(s, lut[q]);
+                        if (j < nv) piece |= q << (T::kBits * j);
+                    }
+                } else {
+                    const float4 rr = rnd24x4(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                    const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t q = degenerate ? 0u : quantise(v[4 * r + j], s, rv[j], kHalfL, (int)kL);
+                        cv[j] = __fmul_rn(s, lut[q]);
+                        if (j < nv) piece |= q << (T::kBits * j);
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) dn[j] = __fadd_rn(v[4 * r + j], -cv[j]);
+                st_partial(p.delta + row + e0, make_float4(dn[0], dn[1], dn[2], dn[3]), nv);
+                *reinterpret_cast<float4*>(cval_mine + e0) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+            }
+            uint32_t word = piece << ((4 * T::kBits * (lane % T::kLanesPerWord)) & 31);
+#pragma unroll
+            for (int o = 1; o < T::kLanesPerWord; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
+            if ((lane % T::kLanesPerWord) == 0 && e0 < live_len)
+                p.codes[code_row + f / T::kLanesPerWord] = word;
+        }
+        if (!p.prescaled && alive && wg == 0 && lane == 0)
+            p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+
+        __syncthreads();       // C[v] of every node of this tile is in shared memory
+        if (abort_sm[buf]) break;
+
+        // ---- phase C: local update from the neighbours' C[v] ---------------
+        float acc[E];
+#pragma unroll
+        for (int t = 0; t < E; ++t) acc[t] = 0.0f;
+        const int e_beg = rp[node], e_end = rp[node + 1];
+        for (int e = e_beg; e < e_end; ++e) {
+            const float w = wp[e];
+            const float* cn = cval + (size_t)cj[e] * p.tile + seg0;
+#pragma unroll
+            for (int r = 0; r < V; ++r) {
+                const int e0 = 4 * (32 * r + lane);
+                if (!full && e0 >= live_len) continue;
+                const float4 c4 = *reinterpret_cast<const float4*>(cn + e0);
+                acc[4 * r + 0] = __fmaf_rn(w, c4.x, acc[4 * r + 0]);
+                acc[4 * r + 1] = __fmaf_rn(w, c4.y, acc[4 * r + 1]);
+                acc[4 * r + 2] = __fmaf_rn(w, c4.z, acc[4 * r + 2]);
+                acc[4 * r + 3] = __fmaf_rn(w, c4.w, acc[4 * r + 3]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < V; ++r) {
+            const int e0 = 4 * (32 * r + lane);
+            const int nv = full ? 4 : min(max(live_len - e0, 0), 4);
+            if (nv > 0)
+                st_partial(p.x + row + e0,
+                           make_float4(__fmaf_rn(p.eta, acc[4 * r + 0], h[4 * r + 0]),
+                                       __fmaf_rn(p.eta, acc[4 * r + 1], h[4 * r + 1]),
+                                       __fmaf_rn(p.eta, acc[4 * r + 2], h[4 * r + 2]),
+                                       __fmaf_rn(p.eta, acc[4 * r + 3], h[4 * r + 3])), nv);
+        }
+        buf ^= 1;
+    }
+    // Leaving early (error path): let the copy that is still in flight land
+    // before the block's shared memory is given away.
+    if (pending) (void)mbar_wait_bounded(bar, parity);
+}
+
+template <int CODE, int NOISE, int E>
+cudaError_t launch_tma_one(const LaunchShape& sh, const StepParams& p, cudaStream_t stream) {
+    if (sh.block.x <= 512) {
+        auto kern = ds_fused_tma_kernel<CODE, NOISE, E, 512>;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem);
+        if (e != cudaSuccess) return e;
+        kern<<<sh.grid, sh.block, sh.smem, stream>>>(p);
+    } else {
+        auto kern = ds_fused_tma_kernel<CODE, NOISE, E, 1024>;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem);
+        if (e != cudaSuccess) return e;
+        kern<<<sh.grid, sh.block, sh.smem, stream>>>(p);
+    }
+    return cudaGetLastError();
+}
+
+template <int CODE>
+cudaError_t launch_tma_code(const LaunchShape& sh, const StepParams& p, cudaStream_t stream) {
+#define DS_TMA_CASE(NZ, EE) \
+    if (sh.noise == NZ && sh.elems_per_lane == EE) return launch_tma_one<CODE, NZ, EE>(sh, p, stream);
+    DS_TMA_CASE(NOISE_NONE, 4) DS_TMA_CASE(NOISE_NONE, 8) DS_TMA_CASE(NOISE_NONE, 16)
+    DS_TMA_CASE(NOISE_GAUSS, 4) DS_TMA_CASE(NOISE_GAUSS, 8) DS_TMA_CASE(NOISE_GAUSS, 16)
+    DS_TMA_CASE(NOISE_T3, 4) DS_TMA_CASE(NOISE_T3, 8) DS_TMA_CASE(NOISE_T3, 16)
+#undef DS_TMA_CASE
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace ds

@@ -35,6 +35,7 @@ struct StepParams {
     float* scales;
     int64_t scales_pitch;
     double* partials;         // [n][tiles], per-node-scale reduction
+    int* error_flag;          // set to 1 by a kernel whose bounded wait ran out
     float sigma;
     float neg_gamma;
     float eta;
@@ -56,6 +57,7 @@ struct LaunchShape {
 
 // Launchers (defined in the kernel translation units).
 cudaError_t launch_column_fused(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
+cudaError_t launch_fused_tma(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_column_compress(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_column_reduce(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_finalize_scales(const StepParams& p, int code, cudaStream_t stream);

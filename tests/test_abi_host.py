@@ -37,8 +37,8 @@ def test_library_exports_every_declared_symbol():
 
 def test_strerror():
     assert B.ds_strerror(B.DS_OK) == "ok"
-    seen = {B.ds_strerror(s) for s in range(0, 11)}
-    assert len(seen) == 11
+    seen = {B.ds_strerror(s) for s in range(0, 12)}
+    assert len(seen) == 12
 
 
 def test_workspace_size():
@@ -161,4 +161,5 @@ def test_null_handles():
     assert L.ds_get_info(None, None) == B.DS_ERR_NULL
     assert L.ds_codes(None, None, None, None, None) == B.DS_ERR_NULL
     assert L.ds_noise(None, 1, 1, 1, 0, 0, 0, 0, None) == B.DS_ERR_NULL
+    assert L.ds_sync(None, None) == B.DS_ERR_NULL
     L.ds_destroy(None)
