@@ -170,6 +170,7 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=sorted(I.WORKLOADS))
     ap.add_argument("--size", type=int, default=0, help="override N (parameters per node)")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "fused_ldg", "split"])
+    ap.add_argument("--elems-per-lane", type=int, default=0, help="tuning knob (0 = library default)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-cols", type=int, default=1 << 24,
@@ -210,6 +211,8 @@ def main():
     ds = B.DeepSqueeze(g, w.N, ld, w.comp_kind, w.bits, w.chunk, device=dev)
     ds.ds_set_path({"auto": B.DS_PATH_AUTO, "fused": B.DS_PATH_FUSED, "fused_ldg": B.DS_PATH_FUSED_LDG,
                     "split": B.DS_PATH_SPLIT}[args.path])
+    if args.elems_per_lane:
+        ds.ds_tune(args.elems_per_lane)
     info = ds.ds_get_info()
     a = torch.from_numpy(a_h).to(dev)
     c = torch.from_numpy(c_h).to(dev)

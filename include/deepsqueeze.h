@@ -185,6 +185,13 @@ ds_status ds_codes(ds_ctx *ctx, const uint32_t **codes, int64_t *code_pitch_word
  * DS_PATH_FUSED is asked for a shape it cannot take. */
 ds_status ds_set_path(ds_ctx *ctx, int32_t path);
 
+/* Tuning knob: elements a lane keeps in registers per (node, chunk): 4, 8 or 16
+ * (0 = the library's choice).  Fewer elements per lane mean more warps per
+ * chunk.  Re-plans every path; a path the new shape cannot take falls back as
+ * DS_PATH_AUTO describes.  DS_ERR_UNSUPPORTED (nothing changed) if not even the
+ * two-kernel path can take it.  Results do not depend on it. */
+ds_status ds_tune(ds_ctx *ctx, int32_t elems_per_lane);
+
 /* Launch geometry of the current path (host-only). */
 ds_status ds_get_info(const ds_ctx *ctx, ds_info *info);
 

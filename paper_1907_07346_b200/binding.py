@@ -24,7 +24,7 @@ DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 
 EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_host", "ds_codes", "ds_set_path",
-           "ds_get_info", "ds_sync", "ds_noise", "ds_destroy", "ds_strerror"]
+           "ds_tune", "ds_get_info", "ds_sync", "ds_noise", "ds_destroy", "ds_strerror"]
 
 
 class ds_graph(C.Structure):
@@ -76,6 +76,8 @@ def lib():
         L.ds_codes.restype = C.c_int
         L.ds_set_path.argtypes = [C.c_void_p, C.c_int32]
         L.ds_set_path.restype = C.c_int
+        L.ds_tune.argtypes = [C.c_void_p, C.c_int32]
+        L.ds_tune.restype = C.c_int
         L.ds_get_info.argtypes = [C.c_void_p, C.POINTER(ds_info)]
         L.ds_get_info.restype = C.c_int
         L.ds_sync.argtypes = [C.c_void_p, C.c_void_p]
@@ -152,6 +154,9 @@ class DeepSqueeze:
 
     def ds_set_path(self, path: int):
         _check(lib().ds_set_path(self.ctx, path), "ds_set_path")
+
+    def ds_tune(self, elems_per_lane: int):
+        _check(lib().ds_tune(self.ctx, elems_per_lane), "ds_tune")
 
     def ds_get_info(self) -> ds_info:
         info = ds_info()

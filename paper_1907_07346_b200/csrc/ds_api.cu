@@ -90,15 +90,15 @@ struct Plan {
     size_t smem = 0;
 };
 
-void pick_lane_shape(int64_t tile, int* E, int* G) {
-    *E = (tile >= 512) ? 16 : (tile >= 256) ? 8 : 4;
+void pick_lane_shape(int64_t tile, int force_e, int* E, int* G) {
+    *E = (force_e > 0) ? force_e : (tile >= 512) ? 16 : (tile >= 256) ? 8 : 4;
     *G = (int)((tile + 32 * (*E) - 1) / (32 * (*E)));
 }
 
-Plan plan_column(int mode, const Shape& sh, int32_t n, int32_t nnz) {
+Plan plan_column(int mode, const Shape& sh, int32_t n, int32_t nnz, int force_e = 0) {
     Plan pl;
     int E, G;
-    pick_lane_shape(sh.tile, &E, &G);
+    pick_lane_shape(sh.tile, force_e, &E, &G);
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
     if (G > 32) return pl;
@@ -121,10 +121,10 @@ Plan plan_column(int mode, const Shape& sh, int32_t n, int32_t nnz) {
     return pl;
 }
 
-Plan plan_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms) {
+Plan plan_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int force_e = 0) {
     Plan pl;
     int E, G;
-    pick_lane_shape(sh.tile, &E, &G);
+    pick_lane_shape(sh.tile, force_e, &E, &G);
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
     if (sh.code == CODE_ID32 || (int64_t)n * G > 32 || num_sms < 1) return pl;
@@ -300,6 +300,19 @@ ds_status ds_set_path(ds_ctx* ctx, int32_t path) {
     if (path == DS_PATH_FUSED && !ctx->fused.ok && !ctx->tma.ok) return DS_ERR_UNSUPPORTED;
     if (path == DS_PATH_FUSED_LDG && !ctx->fused.ok) return DS_ERR_UNSUPPORTED;
     ctx->path_req = path;
+    return DS_OK;
+}
+
+ds_status ds_tune(ds_ctx* ctx, int32_t elems_per_lane) {
+    if (!ctx) return DS_ERR_NULL;
+    if (elems_per_lane != 0 && elems_per_lane != 4 && elems_per_lane != 8 && elems_per_lane != 16)
+        return DS_ERR_ARG;
+    const Plan compress = plan_column(MODE_COMPRESS, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
+    if (!compress.ok) return DS_ERR_UNSUPPORTED;
+    ctx->compress = compress;
+    ctx->reduce = plan_column(MODE_REDUCE, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
+    ctx->tma = plan_tma(ctx->sh, ctx->n, ctx->nnz, ctx->num_sms, elems_per_lane);
+    ctx->fused = plan_column(MODE_FUSED, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
     return DS_OK;
 }
 

@@ -21,6 +21,8 @@
 // storing; the block leaves the tile loop together at the next barrier.
 #pragma once
 
+#include <type_traits>
+
 #include "ds_column_kernel.cuh"
 
 namespace ds {
@@ -166,156 +168,162 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
         const int live_len = alive ? seg_len : 0;
         const bool full = (live_len == SEG);
 
-        // ---- phase A: slot -> registers, local step, scale partial ---------
-        float h[E], v[E];
-        double sum = 0.0;
-        float mx = 0.0f;
-#pragma unroll
-        for (int r = 0; r < V; ++r) {
-            const int e0 = 4 * (32 * r + lane);              // offset inside the segment
-            const int nv = full ? 4 : min(max(live_len - e0, 0), 4);
-            if (nv > 0) {
-                const float4 x4 = *reinterpret_cast<const float4*>(slot + 0 * SEG + e0);
-                const float4 d4 = *reinterpret_cast<const float4*>(slot + 1 * SEG + e0);
-                const float4 a4 = *reinterpret_cast<const float4*>(slot + 2 * SEG + e0);
-                const float4 c4 = *reinterpret_cast<const float4*>(slot + 3 * SEG + e0);
-                const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
-                local_step(x4.x, d4.x, a4.x, c4.x, z4.x, p.sigma, p.neg_gamma, h[4 * r + 0], v[4 * r + 0]);
-                local_step(x4.y, d4.y, a4.y, c4.y, z4.y, p.sigma, p.neg_gamma, h[4 * r + 1], v[4 * r + 1]);
-                local_step(x4.z, d4.z, a4.z, c4.z, z4.z, p.sigma, p.neg_gamma, h[4 * r + 2], v[4 * r + 2]);
-                local_step(x4.w, d4.w, a4.w, c4.w, z4.w, p.sigma, p.neg_gamma, h[4 * r + 3], v[4 * r + 3]);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    if (j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
-                    if constexpr (T::kSign) sum += (double)fabsf(v[4 * r + j]);
-                    else mx = fmaxf(mx, fabsf(v[4 * r + j]));
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
-            }
-        }
-        // the slot is in registers: refill it with the segment of the next tile
-        __syncwarp();
-        {
-            const int64_t next = col + gridDim.x;
-            pending = (next < p.tiles) ? issue(next) : false;
-        }
-
-        // ---- scale of the (node, tile) -----------------------------------
-        float s;
-        if (p.prescaled) {
-            s = p.scales[(size_t)node * (size_t)p.scales_pitch];
-        } else {
-            double part;
-            if constexpr (T::kSign) part = warp_sum(sum);
-            else part = (double)__uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
-            if (G > 1) {
-                double* red = reinterpret_cast<double*>(smem + L.red_off);
-                if (lane == 0) red[warp] = part;
-                __syncthreads();
-                part = 0.0;
-                for (int w = 0; w < G; ++w) {
-                    const double t = red[node * G + w];
-                    if constexpr (T::kSign) part += t;
-                    else part = fmax(part, t);
-                }
-            }
-            if constexpr (T::kSign) {
-                s = (float)(part / (double)m_len);
-            } else {
-                s = (float)part;
-                if (s == 0.0f || !(fabsf(s) <= 3.402823466e+38f)) s = 0.0f;
-            }
-        }
-        const bool degenerate = (!T::kSign && s == 0.0f);
-        const bool fast = T::kLut && s >= 0x1p-60f && s <= 0x1p+60f;
-        const float inv_s = fast ? __fdiv_rn(1.0f, s) : 0.0f;
-        const size_t code_row = (size_t)node * (size_t)p.code_pitch + (size_t)(((k0 + seg0) * T::kBits) >> 5);
-        float* cval_mine = cval + (size_t)node * p.tile + seg0;
-
-        // ---- phase B: compress, residual, pack -----------------------------
-#pragma unroll
-        for (int r = 0; r < V; ++r) {
-            const int f = 32 * r + lane;                     // float4 index inside the segment
-            const int e0 = 4 * f;
-            const int nv = full ? 4 : min(max(live_len - e0, 0), 4);
-            uint32_t piece = 0u;
-            if (nv > 0) {
-                float dn[4], cv[4];
-                if constexpr (T::kSign) {
-#pragma unroll
+        auto tile_body = [&](auto full_tag) -> bool {
+            constexpr bool FULL = decltype(full_tag)::value;
+            // ---- phase A: slot -> registers, local step, scale partial ---------
+            float h[E], v[E];
+            double sum = 0.0;
+            float mx = 0.0f;
+    #pragma unroll
+            for (int r = 0; r < V; ++r) {
+                const int e0 = 4 * (32 * r + lane);              // offset inside the segment
+                const int nv = FULL ? 4 : min(max(live_len - e0, 0), 4);
+                if (nv > 0) {
+                    const float4 x4 = *reinterpret_cast<const float4*>(slot + 0 * SEG + e0);
+                    const float4 d4 = *reinterpret_cast<const float4*>(slot + 1 * SEG + e0);
+                    const float4 a4 = *reinterpret_cast<const float4*>(slot + 2 * SEG + e0);
+                    const float4 c4 = *reinterpret_cast<const float4*>(slot + 3 * SEG + e0);
+                    const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                    local_step(x4.x, d4.x, a4.x, c4.x, z4.x, p.sigma, p.neg_gamma, h[4 * r + 0], v[4 * r + 0]);
+                    local_step(x4.y, d4.y, a4.y, c4.y, z4.y, p.sigma, p.neg_gamma, h[4 * r + 1], v[4 * r + 1]);
+                    local_step(x4.z, d4.z, a4.z, c4.z, z4.z, p.sigma, p.neg_gamma, h[4 * r + 2], v[4 * r + 2]);
+                    local_step(x4.w, d4.w, a4.w, c4.w, z4.w, p.sigma, p.neg_gamma, h[4 * r + 3], v[4 * r + 3]);
+    #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint32_t bit = (v[4 * r + j] >= 0.0f) ? 1u : 0u;
-                        cv[j] = bit ? s : -s;
-                        if (j < nv) piece |= bit << j;
-                    }
-                } else if (fast) {
-                    const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
-                    const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t q = quantise_recip(v[4 * r + j], s, inv_s, rv[j], kHalfL, (int)kL);
-                        cv[j] = __fmul_rn(s, lut[q]);
-                        if (j < nv) piece |= q << (T::kBits * j);
+                        if (!FULL && j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
+                        if constexpr (T::kSign) sum += (double)fabsf(v[4 * r + j]);
+                        else mx = fmaxf(mx, fabsf(v[4 * r + j]));
                     }
                 } else {
-                    const float4 rr = rnd24x4(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
-                    const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t q = degenerate ? 0u : quantise(v[4 * r + j], s, rv[j], kHalfL, (int)kL);
-                        cv[j] = __fmul_rn(s, lut[q]);
-                        if (j < nv) piece |= q << (T::kBits * j);
+    #pragma unroll
+                    for (int j = 0; j < 4; ++j) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
+                }
+            }
+            // the slot is in registers: refill it with the segment of the next tile
+            __syncwarp();
+            {
+                const int64_t next = col + gridDim.x;
+                pending = (next < p.tiles) ? issue(next) : false;
+            }
+
+            // ---- scale of the (node, tile) -----------------------------------
+            float s;
+            if (p.prescaled) {
+                s = p.scales[(size_t)node * (size_t)p.scales_pitch];
+            } else {
+                double part;
+                if constexpr (T::kSign) part = warp_sum(sum);
+                else part = (double)__uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
+                if (G > 1) {
+                    double* red = reinterpret_cast<double*>(smem + L.red_off);
+                    if (lane == 0) red[warp] = part;
+                    __syncthreads();
+                    part = 0.0;
+                    for (int w = 0; w < G; ++w) {
+                        const double t = red[node * G + w];
+                        if constexpr (T::kSign) part += t;
+                        else part = fmax(part, t);
                     }
                 }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) dn[j] = __fadd_rn(v[4 * r + j], -cv[j]);
-                st_partial(p.delta + row + e0, make_float4(dn[0], dn[1], dn[2], dn[3]), nv);
-                *reinterpret_cast<float4*>(cval_mine + e0) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+                if constexpr (T::kSign) {
+                    s = (float)(part / (double)m_len);
+                } else {
+                    s = (float)part;
+                    if (s == 0.0f || !(fabsf(s) <= 3.402823466e+38f)) s = 0.0f;
+                }
             }
-            uint32_t word = piece << ((4 * T::kBits * (lane % T::kLanesPerWord)) & 31);
-#pragma unroll
-            for (int o = 1; o < T::kLanesPerWord; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
-            if ((lane % T::kLanesPerWord) == 0 && e0 < live_len)
-                p.codes[code_row + f / T::kLanesPerWord] = word;
-        }
-        if (!p.prescaled && alive && wg == 0 && lane == 0)
-            p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+            const bool degenerate = (!T::kSign && s == 0.0f);
+            const bool fast = T::kLut && s >= 0x1p-60f && s <= 0x1p+60f;
+            const float inv_s = fast ? __fdiv_rn(1.0f, s) : 0.0f;
+            const size_t code_row = (size_t)node * (size_t)p.code_pitch + (size_t)(((k0 + seg0) * T::kBits) >> 5);
+            float* cval_mine = cval + (size_t)node * p.tile + seg0;
 
-        __syncthreads();       // C[v] of every node of this tile is in shared memory
-        if (abort_sm[buf]) break;
+            // ---- phase B: compress, residual, pack -----------------------------
+    #pragma unroll
+            for (int r = 0; r < V; ++r) {
+                const int f = 32 * r + lane;                     // float4 index inside the segment
+                const int e0 = 4 * f;
+                const int nv = FULL ? 4 : min(max(live_len - e0, 0), 4);
+                uint32_t piece = 0u;
+                if (nv > 0) {
+                    float dn[4], cv[4];
+                    if constexpr (T::kSign) {
+    #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t bit = (v[4 * r + j] >= 0.0f) ? 1u : 0u;
+                            cv[j] = bit ? s : -s;
+                            if (FULL || j < nv) piece |= bit << j;
+                        }
+                    } else if (fast) {
+                        const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                        const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
+    #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t q = quantise_recip(v[4 * r + j], s, inv_s, rv[j], kHalfL, (int)kL);
+                            cv[j] = __fmul_rn(s, lut[q]);
+                            if (FULL || j < nv) piece |= q << (T::kBits * j);
+                        }
+                    } else {
+                        const float4 rr = rnd24x4(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                        const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
+    #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t q = degenerate ? 0u : quantise(v[4 * r + j], s, rv[j], kHalfL, (int)kL);
+                            cv[j] = __fmul_rn(s, lut[q]);
+                            if (FULL || j < nv) piece |= q << (T::kBits * j);
+                        }
+                    }
+    #pragma unroll
+                    for (int j = 0; j < 4; ++j) dn[j] = __fadd_rn(v[4 * r + j], -cv[j]);
+                    st_partial(p.delta + row + e0, make_float4(dn[0], dn[1], dn[2], dn[3]), nv);
+                    *reinterpret_cast<float4*>(cval_mine + e0) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+                }
+                uint32_t word = piece << ((4 * T::kBits * (lane % T::kLanesPerWord)) & 31);
+    #pragma unroll
+                for (int o = 1; o < T::kLanesPerWord; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
+                if ((lane % T::kLanesPerWord) == 0 && (FULL || e0 < live_len))
+                    p.codes[code_row + f / T::kLanesPerWord] = word;
+            }
+            if (!p.prescaled && alive && wg == 0 && lane == 0)
+                p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
 
-        // ---- phase C: local update from the neighbours' C[v] ---------------
-        float acc[E];
-#pragma unroll
-        for (int t = 0; t < E; ++t) acc[t] = 0.0f;
-        const int e_beg = rp[node], e_end = rp[node + 1];
-        for (int e = e_beg; e < e_end; ++e) {
-            const float w = wp[e];
-            const float* cn = cval + (size_t)cj[e] * p.tile + seg0;
-#pragma unroll
+            __syncthreads();       // C[v] of every node of this tile is in shared memory
+            if (abort_sm[buf]) return true;
+
+            // ---- phase C: local update from the neighbours' C[v] ---------------
+            float acc[E];
+    #pragma unroll
+            for (int t = 0; t < E; ++t) acc[t] = 0.0f;
+            const int e_beg = rp[node], e_end = rp[node + 1];
+            for (int e = e_beg; e < e_end; ++e) {
+                const float w = wp[e];
+                const float* cn = cval + (size_t)cj[e] * p.tile + seg0;
+    #pragma unroll
+                for (int r = 0; r < V; ++r) {
+                    const int e0 = 4 * (32 * r + lane);
+                    if (!FULL && e0 >= live_len) continue;
+                    const float4 c4 = *reinterpret_cast<const float4*>(cn + e0);
+                    acc[4 * r + 0] = __fmaf_rn(w, c4.x, acc[4 * r + 0]);
+                    acc[4 * r + 1] = __fmaf_rn(w, c4.y, acc[4 * r + 1]);
+                    acc[4 * r + 2] = __fmaf_rn(w, c4.z, acc[4 * r + 2]);
+                    acc[4 * r + 3] = __fmaf_rn(w, c4.w, acc[4 * r + 3]);
+                }
+            }
+    #pragma unroll
             for (int r = 0; r < V; ++r) {
                 const int e0 = 4 * (32 * r + lane);
-                if (!full && e0 >= live_len) continue;
-                const float4 c4 = *reinterpret_cast<const float4*>(cn + e0);
-                acc[4 * r + 0] = __fmaf_rn(w, c4.x, acc[4 * r + 0]);
-                acc[4 * r + 1] = __fmaf_rn(w, c4.y, acc[4 * r + 1]);
-                acc[4 * r + 2] = __fmaf_rn(w, c4.z, acc[4 * r + 2]);
-                acc[4 * r + 3] = __fmaf_rn(w, c4.w, acc[4 * r + 3]);
+                const int nv = FULL ? 4 : min(max(live_len - e0, 0), 4);
+                if (nv > 0)
+                    st_partial(p.x + row + e0,
+                               make_float4(__fmaf_rn(p.eta, acc[4 * r + 0], h[4 * r + 0]),
+                                           __fmaf_rn(p.eta, acc[4 * r + 1], h[4 * r + 1]),
+                                           __fmaf_rn(p.eta, acc[4 * r + 2], h[4 * r + 2]),
+                                           __fmaf_rn(p.eta, acc[4 * r + 3], h[4 * r + 3])), nv);
             }
-        }
-#pragma unroll
-        for (int r = 0; r < V; ++r) {
-            const int e0 = 4 * (32 * r + lane);
-            const int nv = full ? 4 : min(max(live_len - e0, 0), 4);
-            if (nv > 0)
-                st_partial(p.x + row + e0,
-                           make_float4(__fmaf_rn(p.eta, acc[4 * r + 0], h[4 * r + 0]),
-                                       __fmaf_rn(p.eta, acc[4 * r + 1], h[4 * r + 1]),
-                                       __fmaf_rn(p.eta, acc[4 * r + 2], h[4 * r + 2]),
-                                       __fmaf_rn(p.eta, acc[4 * r + 3], h[4 * r + 3])), nv);
-        }
+            return false;
+        };
+        const bool aborted = full ? tile_body(std::true_type{}) : tile_body(std::false_type{});
+        if (aborted) break;
         buf ^= 1;
     }
     // Leaving early (error path): let the copy that is still in flight land
