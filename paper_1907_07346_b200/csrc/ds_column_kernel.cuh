@@ -121,10 +121,7 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
             const float4 a4 = ld4(p.a + row + e0);
             const float4 c4 = ld4(p.c + row + e0);
             const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + e0));
-            local_step(x4.x, d4.x, a4.x, c4.x, z4.x, p.sigma, p.neg_gamma, h[4 * r + 0], v[4 * r + 0]);
-            local_step(x4.y, d4.y, a4.y, c4.y, z4.y, p.sigma, p.neg_gamma, h[4 * r + 1], v[4 * r + 1]);
-            local_step(x4.z, d4.z, a4.z, c4.z, z4.z, p.sigma, p.neg_gamma, h[4 * r + 2], v[4 * r + 2]);
-            local_step(x4.w, d4.w, a4.w, c4.w, z4.w, p.sigma, p.neg_gamma, h[4 * r + 3], v[4 * r + 3]);
+            local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 if (!FULL && j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }

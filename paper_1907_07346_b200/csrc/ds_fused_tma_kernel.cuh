@@ -184,10 +184,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     const float4 a4 = *reinterpret_cast<const float4*>(slot + 2 * SEG + e0);
                     const float4 c4 = *reinterpret_cast<const float4*>(slot + 3 * SEG + e0);
                     const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
-                    local_step(x4.x, d4.x, a4.x, c4.x, z4.x, p.sigma, p.neg_gamma, h[4 * r + 0], v[4 * r + 0]);
-                    local_step(x4.y, d4.y, a4.y, c4.y, z4.y, p.sigma, p.neg_gamma, h[4 * r + 1], v[4 * r + 1]);
-                    local_step(x4.z, d4.z, a4.z, c4.z, z4.z, p.sigma, p.neg_gamma, h[4 * r + 2], v[4 * r + 2]);
-                    local_step(x4.w, d4.w, a4.w, c4.w, z4.w, p.sigma, p.neg_gamma, h[4 * r + 3], v[4 * r + 3]);
+                    local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
     #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         if (!FULL && j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
@@ -256,13 +253,15 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                         }
                     } else if (fast) {
                         const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
-                        const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
-    #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t q = quantise_recip(v[4 * r + j], s, inv_s, rv[j], kHalfL, (int)kL);
-                            cv[j] = __fmul_rn(s, lut[q]);
-                            if (FULL || j < nv) piece |= q << (T::kBits * j);
-                        }
+                        uint32_t q[4];
+                        quantise_recip2(v[4 * r + 0], v[4 * r + 1], s, inv_s, rr.x, rr.y, kHalfL, (int)kL, q[0], q[1]);
+                        quantise_recip2(v[4 * r + 2], v[4 * r + 3], s, inv_s, rr.z, rr.w, kHalfL, (int)kL, q[2], q[3]);
+                        const float2 ca = __fmul2_rn(splat(s), make_float2(lut[q[0]], lut[q[1]]));
+                        const float2 cb = __fmul2_rn(splat(s), make_float2(lut[q[2]], lut[q[3]]));
+                        cv[0] = ca.x; cv[1] = ca.y; cv[2] = cb.x; cv[3] = cb.y;
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (FULL || j < nv) piece |= q[j] << (T::kBits * j);
                     } else {
                         const float4 rr = rnd24x4(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
                         const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
@@ -273,8 +272,11 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                             if (FULL || j < nv) piece |= q << (T::kBits * j);
                         }
                     }
-    #pragma unroll
-                    for (int j = 0; j < 4; ++j) dn[j] = __fadd_rn(v[4 * r + j], -cv[j]);
+                        {
+                        const float2 da = __fadd2_rn(make_float2(v[4 * r + 0], v[4 * r + 1]), make_float2(-cv[0], -cv[1]));
+                        const float2 db = __fadd2_rn(make_float2(v[4 * r + 2], v[4 * r + 3]), make_float2(-cv[2], -cv[3]));
+                        dn[0] = da.x; dn[1] = da.y; dn[2] = db.x; dn[3] = db.y;
+                    }
                     st_partial(p.delta + row + e0, make_float4(dn[0], dn[1], dn[2], dn[3]), nv);
                     *reinterpret_cast<float4*>(cval_mine + e0) = make_float4(cv[0], cv[1], cv[2], cv[3]);
                 }
@@ -303,22 +305,24 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     const int e0 = 4 * (32 * r + lane);
                     if (!FULL && e0 >= live_len) continue;
                     const float4 c4 = *reinterpret_cast<const float4*>(cn + e0);
-                    acc[4 * r + 0] = __fmaf_rn(w, c4.x, acc[4 * r + 0]);
-                    acc[4 * r + 1] = __fmaf_rn(w, c4.y, acc[4 * r + 1]);
-                    acc[4 * r + 2] = __fmaf_rn(w, c4.z, acc[4 * r + 2]);
-                    acc[4 * r + 3] = __fmaf_rn(w, c4.w, acc[4 * r + 3]);
+                    {
+                        const float2 w2 = splat(w);
+                        const float2 aa = __ffma2_rn(w2, make_float2(c4.x, c4.y), make_float2(acc[4 * r + 0], acc[4 * r + 1]));
+                        const float2 ab = __ffma2_rn(w2, make_float2(c4.z, c4.w), make_float2(acc[4 * r + 2], acc[4 * r + 3]));
+                        acc[4 * r + 0] = aa.x; acc[4 * r + 1] = aa.y; acc[4 * r + 2] = ab.x; acc[4 * r + 3] = ab.y;
+                    }
                 }
             }
     #pragma unroll
             for (int r = 0; r < V; ++r) {
                 const int e0 = 4 * (32 * r + lane);
                 const int nv = FULL ? 4 : min(max(live_len - e0, 0), 4);
-                if (nv > 0)
-                    st_partial(p.x + row + e0,
-                               make_float4(__fmaf_rn(p.eta, acc[4 * r + 0], h[4 * r + 0]),
-                                           __fmaf_rn(p.eta, acc[4 * r + 1], h[4 * r + 1]),
-                                           __fmaf_rn(p.eta, acc[4 * r + 2], h[4 * r + 2]),
-                                           __fmaf_rn(p.eta, acc[4 * r + 3], h[4 * r + 3])), nv);
+                if (nv > 0) {
+                    const float2 et = splat(p.eta);
+                    const float2 xa = __ffma2_rn(et, make_float2(acc[4 * r + 0], acc[4 * r + 1]), make_float2(h[4 * r + 0], h[4 * r + 1]));
+                    const float2 xb = __ffma2_rn(et, make_float2(acc[4 * r + 2], acc[4 * r + 3]), make_float2(h[4 * r + 2], h[4 * r + 3]));
+                    st_partial(p.x + row + e0, make_float4(xa.x, xa.y, xb.x, xb.y), nv);
+                }
             }
             return false;
         };
