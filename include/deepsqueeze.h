@@ -208,6 +208,42 @@ ds_status ds_sync(ds_ctx *ctx, void *cuda_stream);
 ds_status ds_noise(float *out, int32_t n, int64_t N, int64_t ld_out, int32_t which,
                    int32_t noise, uint64_t seed, uint64_t step, void *cuda_stream);
 
+/* Per-node compressor scales with NO device allocation and no workspace.
+ * (The paper has no counterpart: this entry point exists for the callers
+ * described below, not for a step of Algorithm 1.)
+ *
+ * Some callers cannot obtain device memory when they call: code running inside
+ * a process whose framework has already claimed the whole GPU for its own
+ * memory pool, code on a path where an allocation would synchronise the device
+ * and stall a latency-critical loop, or code that simply is not allowed to call
+ * the allocator (plug-ins, callbacks).  For them this computes, for every node
+ * i, the scale of the error-compensated variable v_i = x_i - gamma g_i + delta_i
+ * over the WHOLE row -- what ds_step uses when the compressor has chunk = 0:
+ *     comp_kind = DS_COMP_SIGN1_L1              s_i = (sum_k |v_ik|) / N
+ *     comp_kind = DS_COMP_UNIFORM_STOCH_MAXABS  s_i = max_k |v_ik|  (0 if not finite)
+ * and writes it to scales_out[i] (device, n floats).  x, delta, gp->a, gp->c are
+ * device [n][ld] arrays as for ds_step and are only read.
+ *
+ * The reduction's scratch is a fixed array inside the library
+ * (DS_NOALLOC_MAX_PARTIALS binary64 partials plus a 1 KiB table, 544 KiB, held on
+ * every GPU that loads the library until the process exits).  Consequences:
+ *   - sizes with n * ceil(N / 512) > DS_NOALLOC_MAX_PARTIALS are rejected with
+ *     DS_ERR_WORKSPACE;
+ *   - all calls on one GPU share the array, so two calls whose kernels can
+ *     overlap on the GPU (different streams, no dependency) race; serialise them;
+ *   - the array keeps the previous call's contents, which is harmless: each call
+ *     overwrites every partial it later reads;
+ *   - the first call on each device looks up the array's device address (with
+ *     that device current); make that first call before starting any stream
+ *     capture.
+ * The call allocates nothing: no cudaMalloc, cudaFree or allocating library
+ * routine.  It only enqueues two kernels on cuda_stream. */
+#define DS_NOALLOC_MAX_PARTIALS 65536
+ds_status ds_node_scales_noalloc(float *scales_out, const float *x, const float *delta,
+                                 const ds_grad_params *gp, float gamma, int32_t n, int64_t N,
+                                 int64_t ld, int32_t comp_kind, uint64_t seed, uint64_t step,
+                                 void *cuda_stream);
+
 void ds_destroy(ds_ctx *ctx);
 
 const char *ds_strerror(ds_status status);

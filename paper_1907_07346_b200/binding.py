@@ -24,7 +24,8 @@ DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 
 EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_host", "ds_codes", "ds_set_path",
-           "ds_tune", "ds_get_info", "ds_sync", "ds_noise", "ds_destroy", "ds_strerror"]
+           "ds_tune", "ds_get_info", "ds_sync", "ds_noise", "ds_node_scales_noalloc",
+           "ds_destroy", "ds_strerror"]
 
 
 class ds_graph(C.Structure):
@@ -85,6 +86,10 @@ def lib():
         L.ds_noise.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
                                C.c_uint64, C.c_uint64, C.c_void_p]
         L.ds_noise.restype = C.c_int
+        L.ds_node_scales_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ds_grad_params),
+                                             C.c_float, C.c_int32, C.c_int64, C.c_int64, C.c_int32,
+                                             C.c_uint64, C.c_uint64, C.c_void_p]
+        L.ds_node_scales_noalloc.restype = C.c_int
         L.ds_destroy.argtypes = [C.c_void_p]
         L.ds_destroy.restype = None
         L.ds_strerror.argtypes = [C.c_int]
@@ -233,3 +238,16 @@ def ds_noise(out, n: int, N: int, which: int, noise: int, seed: int, step: int, 
     s = torch.cuda.current_stream(out.device) if stream is None else stream
     _check(lib().ds_noise(out.data_ptr(), n, N, out.shape[1], which, noise, seed, step,
                           C.c_void_p(s.cuda_stream)), "ds_noise")
+
+
+def ds_node_scales_noalloc(scales_out, x, delta, a, c, sigma: float, noise: int, gamma: float,
+                           N: int, comp_kind: int, seed: int, step: int, stream=None) -> int:
+    """Per-node scales into the device tensor scales_out[n] without any device
+    allocation (see include/deepsqueeze.h).  Returns the ds_status."""
+    import torch
+    n, ld = x.shape
+    gp = ds_grad_params(a.data_ptr(), c.data_ptr(), sigma, noise)
+    s = torch.cuda.current_stream(x.device) if stream is None else stream
+    return int(lib().ds_node_scales_noalloc(scales_out.data_ptr(), x.data_ptr(), delta.data_ptr(),
+                                            C.byref(gp), gamma, n, N, ld, comp_kind, seed, step,
+                                            C.c_void_p(s.cuda_stream)))
