@@ -72,7 +72,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -111,6 +111,21 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's device time (every rank gets the same number back)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, updates_per_step: int, steps: int, total_ms: float) -> float:
+    """Updates of all replicas per second of the slowest replica."""
+    return world * updates_per_step * steps / (total_ms * 1e-3)
+
+
 def cpu_baseline(w: I.Workload, a: np.ndarray, c: np.ndarray, sample_cols: int, steps: int = 1,
                  full_N: int | None = None):
     """Time the CPU checker, as it stands, on the first `sample_cols` columns
@@ -118,7 +133,7 @@ def cpu_baseline(w: I.Workload, a: np.ndarray, c: np.ndarray, sample_cols: int, 
     from oracle import oracle as orc
     g = w.build_graph()
     cols = min(sample_cols, w.N)
-    if w.chunk > 0:
+    if w.chunk > 0 and cols < w.N:
         cols = max(w.chunk, cols // w.chunk * w.chunk)
     ld = I.round_up(cols, 4)
     aa = np.zeros((w.n, ld), np.float32)
@@ -165,7 +180,7 @@ def run_reference(args, w: I.Workload):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg3", choices=sorted(I.WORKLOADS))
     ap.add_argument("--size", type=int, default=0, help="override N (parameters per node)")
@@ -173,7 +188,8 @@ def main():
     ap.add_argument("--elems-per-lane", type=int, default=0, help="tuning knob (0 = library default)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-cols", type=int, default=1 << 24,
+    ap.add_argument("--cpu-steps", type=int, default=3, help="steps of the CPU-baseline sample")
+    ap.add_argument("--cpu-cols", type=int, default=1 << 25,
                     help="columns per node of the CPU-baseline sample")
     ap.add_argument("--ref-cols", type=int, default=1 << 21,
                     help="columns per node of each step of --impl reference")
@@ -247,12 +263,9 @@ def main():
     clocks = sampler.stop(t_wall0, t_wall1)
     total_ms = events[0].elapsed_time(events[-1])
     per_step = [events[k].elapsed_time(events[k + 1]) for k in range(args.steps)]
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, dev)
     updates_per_step = w.n * w.N
-    value = world * updates_per_step * args.steps / (total_ms * 1e-3)
+    value = whole_job_value(world, updates_per_step, args.steps, total_ms)
     ds.ds_sync(stream)
     assert torch.isfinite(x).all() and torch.isfinite(delta).all()
 
@@ -290,13 +303,9 @@ def main():
                             x, delta, a, c, stream)
         e1.record(stream)
         barrier()
-        e2e_ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
         arr_bytes = w.n * ld * 4
-        e2e = {"value": world * updates_per_step * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+        e2e = {"value": whole_job_value(world, updates_per_step, args.e2e_steps, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": 4 * arr_bytes, "d2h_bytes_per_step": 2 * arr_bytes,
                "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
                "entry_point": "ds_step_host (pinned host x, delta, a, c in; x, delta out)"}
@@ -304,7 +313,7 @@ def main():
 
     base = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        base, _ = cpu_baseline(w, a_h, c_h, args.cpu_cols, steps=1)
+        base, _ = cpu_baseline(w, a_h, c_h, args.cpu_cols, steps=args.cpu_steps)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
