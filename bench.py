@@ -46,6 +46,24 @@ def algorithmic_bytes_per_update(w: I.Workload) -> float:
     return 24.0 + bits / 8.0 + 4.0 / chunk
 
 
+# DRAM bytes per update of the dominant kernel from the ncu capture summarised in
+# profiles/ds_fused_tma_kernel_cfg3_small_counters.md (dram__bytes_read.sum +
+# dram__bytes_write.sum over one launch of 67,108,864 updates), valid for the
+# kernel sources whose digest is recorded beside it.
+NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59476e9 / 67108864,
+               "sources_sha256": "2244700821305019a93191fee9195e617ad8ec205ae15fad040b46413e7690d3"}
+KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
+
+
+def kernel_sources_digest() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_1907_07346_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -274,9 +292,13 @@ def main():
     b_alg = algorithmic_bytes_per_update(w)
     peak, peak_kind = measured_peak()
     kernel_ms = statistics.mean(per_step)
+    traffic = None      # per launch; null once the kernel sources differ from the profiled ones
+    if (info.path == B.DS_PATH_FUSED and args.workload == NCU_TRAFFIC["workload"] and not args.elems_per_lane
+            and kernel_sources_digest() == NCU_TRAFFIC["sources_sha256"]):
+        traffic = NCU_TRAFFIC["bytes_per_update"] * updates_per_step
     achieved = b_alg * updates_per_step / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None, "peak_source": f"of {peak_kind}",
+                "frac": achieved / peak, "traffic": traffic, "peak_source": f"of {peak_kind}",
                 "kernel": {B.DS_PATH_FUSED: "ds_fused_tma_kernel", B.DS_PATH_FUSED_LDG: "ds_column_kernel (fused)",
                            B.DS_PATH_SPLIT: "ds_column_kernel (compress) + ds_mix_kernel"}[info.path],
                 "algorithmic_bytes_per_update": b_alg,
