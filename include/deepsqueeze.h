@@ -113,7 +113,10 @@ typedef struct {
  *                      inputs are staged by bulk asynchronous copies (TMA); otherwise the
  *                      variant below.
  *   DS_PATH_FUSED_LDG  the fused kernel with direct vector loads and packed codes in shared
- *                      memory (one block per column).
+ *                      memory (one block per column).  When a block cannot hold all nodes of
+ *                      a column at once (many nodes, long chunks) it sweeps them in batches:
+ *                      x - gamma g is parked in x, the codes of the whole column stay in shared
+ *                      memory, and a second sweep re-reads the parked values (from L2) to mix.
  *   DS_PATH_SPLIT      two kernels: compress (x - gamma g written into x, codes to the
  *                      workspace), then mix (each neighbour's packed codes streamed once and
  *                      decoded in registers).  Works for every shape.
@@ -129,6 +132,7 @@ typedef struct {
     int32_t grid_blocks;        /* blocks of the main kernel */
     int64_t chunks_per_row;     /* M = ceil(N / chunk) */
     int64_t code_words_per_row; /* ceil(N * code_bits / 32) */
+    int32_t node_batches;       /* batches of nodes a block sweeps per column (1 = all at once) */
 } ds_info;
 
 /* Bytes of device workspace ds_init needs for this shape (host-only call;

@@ -47,7 +47,8 @@ class ds_hparams(C.Structure):
 class ds_info(C.Structure):
     _fields_ = [("path", C.c_int32), ("launches_per_step", C.c_int32), ("elems_per_lane", C.c_int32),
                 ("warps_per_chunk", C.c_int32), ("block_threads", C.c_int32), ("grid_blocks", C.c_int32),
-                ("chunks_per_row", C.c_int64), ("code_words_per_row", C.c_int64)]
+                ("chunks_per_row", C.c_int64), ("code_words_per_row", C.c_int64),
+                ("node_batches", C.c_int32)]
 
 
 _lib = None

@@ -8,6 +8,7 @@
 
 #include "../../include/deepsqueeze.h"
 #include "ds_fused_tma_kernel.cuh"
+#include "ds_wide_fused_kernel.cuh"
 
 using namespace ds;
 
@@ -140,6 +141,25 @@ Plan plan_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int force_e 
     return pl;
 }
 
+// Fused kernel that sweeps the nodes of a column in batches of nodes_per_block.
+Plan plan_wide(const Shape& sh, int32_t n, int32_t nnz, int force_e = 0) {
+    Plan pl;
+    int E, G;
+    pick_lane_shape(sh.tile, force_e, &E, &G);
+    pl.elems_per_lane = E;
+    pl.warps_per_group = G;
+    if (sh.code == CODE_ID32 || G > 16) return pl;
+    const int npb = std::max(1, std::min<int>(n, 16 / G));
+    pl.nodes_per_block = npb;
+    pl.block = dim3((unsigned)(npb * G * 32));
+    const bool lut = (sh.code != CODE_SIGN);
+    pl.smem = wide_smem_layout(sh.code_bits, lut, npb, G, sh.tile, n, nnz).total;
+    if (pl.smem > (size_t)kMaxSmem) return pl;
+    pl.grid = dim3((unsigned)std::min<int64_t>(sh.tiles, 0x7fffffff));
+    pl.ok = true;
+    return pl;
+}
+
 }  // namespace
 
 struct ds_ctx {
@@ -150,7 +170,7 @@ struct ds_ctx {
     WsLayout ws;
     unsigned char* base;
     int path_req;
-    Plan tma, fused, compress, reduce;
+    Plan tma, fused, wide, compress, reduce;
     int num_sms;
 };
 
@@ -256,6 +276,7 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     ctx->num_sms = sms;
     ctx->tma = plan_tma(sh, n, nnz, sms);
     ctx->fused = plan_column(MODE_FUSED, sh, n, nnz);
+    ctx->wide = plan_wide(sh, n, nnz);
 
     // w'_ij = W_ij - I_ij in binary32; reconstruction levels (2q - L)/L.
     std::vector<float> wprime((size_t)nnz);
@@ -286,19 +307,20 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
 
 void ds_destroy(ds_ctx* ctx) { delete ctx; }
 
-// 2: persistent TMA-staged fused kernel, 1: fused kernel with direct loads, 0: two kernels
+// 2: persistent TMA-staged fused kernel, 1: fused kernel with direct loads,
+// 3: the same in node batches (wide columns), 0: two kernels
 static int fused_kind(const ds_ctx* ctx) {
     if (ctx->path_req == DS_PATH_SPLIT) return 0;
-    if (ctx->path_req == DS_PATH_FUSED_LDG) return ctx->fused.ok ? 1 : 0;
-    if (ctx->tma.ok) return 2;
-    return ctx->fused.ok ? 1 : 0;
+    if (ctx->path_req != DS_PATH_FUSED_LDG && ctx->tma.ok) return 2;
+    if (ctx->fused.ok) return 1;
+    return ctx->wide.ok ? 3 : 0;
 }
 
 ds_status ds_set_path(ds_ctx* ctx, int32_t path) {
     if (!ctx) return DS_ERR_NULL;
     if (path < DS_PATH_AUTO || path > DS_PATH_FUSED_LDG) return DS_ERR_ARG;
-    if (path == DS_PATH_FUSED && !ctx->fused.ok && !ctx->tma.ok) return DS_ERR_UNSUPPORTED;
-    if (path == DS_PATH_FUSED_LDG && !ctx->fused.ok) return DS_ERR_UNSUPPORTED;
+    if (path == DS_PATH_FUSED && !ctx->fused.ok && !ctx->tma.ok && !ctx->wide.ok) return DS_ERR_UNSUPPORTED;
+    if (path == DS_PATH_FUSED_LDG && !ctx->fused.ok && !ctx->wide.ok) return DS_ERR_UNSUPPORTED;
     ctx->path_req = path;
     return DS_OK;
 }
@@ -313,6 +335,7 @@ ds_status ds_tune(ds_ctx* ctx, int32_t elems_per_lane) {
     ctx->reduce = plan_column(MODE_REDUCE, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
     ctx->tma = plan_tma(ctx->sh, ctx->n, ctx->nnz, ctx->num_sms, elems_per_lane);
     ctx->fused = plan_column(MODE_FUSED, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
+    ctx->wide = plan_wide(ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
     return DS_OK;
 }
 
@@ -320,8 +343,9 @@ ds_status ds_get_info(const ds_ctx* ctx, ds_info* info) {
     if (!ctx || !info) return DS_ERR_NULL;
     const int kind = fused_kind(ctx);
     const bool fused = kind != 0;
-    const Plan& pl = (kind == 2) ? ctx->tma : (kind == 1) ? ctx->fused : ctx->compress;
-    info->path = (kind == 2) ? DS_PATH_FUSED : (kind == 1) ? DS_PATH_FUSED_LDG : DS_PATH_SPLIT;
+    const Plan& pl = (kind == 2) ? ctx->tma : (kind == 1) ? ctx->fused : (kind == 3) ? ctx->wide : ctx->compress;
+    info->path = (kind == 2) ? DS_PATH_FUSED : (kind != 0) ? DS_PATH_FUSED_LDG : DS_PATH_SPLIT;
+    info->node_batches = (kind == 3) ? (ctx->n + pl.nodes_per_block - 1) / pl.nodes_per_block : 1;
     info->launches_per_step = (fused ? 1 : 2) + (ctx->sh.per_node ? 2 : 0);
     info->elems_per_lane = pl.elems_per_lane;
     info->warps_per_chunk = pl.warps_per_group;
@@ -391,6 +415,10 @@ ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp,
             p.warps_per_group = ctx->tma.warps_per_group;
             p.nodes_per_block = ctx->tma.nodes_per_block;
             e = launch_fused_tma(shape_of(ctx->tma, MODE_FUSED), p, stream);
+        } else if (kind == 3) {
+            p.warps_per_group = ctx->wide.warps_per_group;
+            p.nodes_per_block = ctx->wide.nodes_per_block;
+            e = launch_fused_wide(shape_of(ctx->wide, MODE_FUSED), p, stream);
         } else if (kind == 1) {
             p.warps_per_group = ctx->fused.warps_per_group;
             p.nodes_per_block = ctx->fused.nodes_per_block;
