@@ -38,12 +38,13 @@ UNIT = "updates/s"
 FALLBACK_HBM_GBS = 6650.0
 
 
-def algorithmic_bytes_per_update(w: I.Workload) -> float:
-    """Read x, delta, a, c (16 B), write x, delta (8 B), write the codes (b/8 B)
-    and one binary32 scale per chunk (4/chunk B)."""
+def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) -> float:
+    """Read x, delta, a, c (16 B; x, delta, g = 12 B when the gradient is given),
+    write x, delta (8 B), write the codes (b/8 B) and one binary32 scale per
+    chunk (4/chunk B)."""
     bits = 32 if w.comp_kind == I.COMP_IDENTITY else (1 if w.comp_kind == I.COMP_SIGN1_L1 else w.bits)
     chunk = w.chunk if w.chunk > 0 else w.N
-    return 24.0 + bits / 8.0 + 4.0 / chunk
+    return (20.0 if given_gradient else 24.0) + bits / 8.0 + 4.0 / chunk
 
 
 # DRAM bytes per update of the dominant kernel from the ncu capture summarised in
@@ -204,6 +205,8 @@ def main():
     ap.add_argument("--size", type=int, default=0, help="override N (parameters per node)")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "fused_ldg", "split"])
     ap.add_argument("--elems-per-lane", type=int, default=0, help="tuning knob (0 = library default)")
+    ap.add_argument("--given-gradient", action="store_true",
+                    help="time ds_step_g (gradient read from memory) instead of the synthetic objective")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-steps", type=int, default=3, help="steps of the CPU-baseline sample")
@@ -259,9 +262,15 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
+    def one_step(k):
+        if args.given_gradient:       # a stands in for the caller's gradient array
+            ds.ds_step_g(x, delta, a, w.gamma, w.eta, w.seed, k, stream)
+        else:
+            ds.ds_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, k, stream)
+
     step_index = 0
     for _ in range(args.warmup):
-        ds.ds_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, step_index, stream)
+        one_step(step_index)
         step_index += 1
     barrier()
 
@@ -273,7 +282,7 @@ def main():
     t_wall0 = time.time()
     events[0].record(stream)
     for k in range(args.steps):
-        ds.ds_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, step_index, stream)
+        one_step(step_index)
         step_index += 1
         events[k + 1].record(stream)
     barrier()
@@ -289,11 +298,11 @@ def main():
 
     # Roofline of the dominant kernel.  On the fused path a step IS one launch
     # of the column kernel, so its average duration is the event time per step.
-    b_alg = algorithmic_bytes_per_update(w)
+    b_alg = algorithmic_bytes_per_update(w, args.given_gradient)
     peak, peak_kind = measured_peak()
     kernel_ms = statistics.mean(per_step)
     traffic = None      # per launch; null once the kernel sources differ from the profiled ones
-    if (info.path == B.DS_PATH_FUSED and args.workload == NCU_TRAFFIC["workload"] and not args.elems_per_lane
+    if (not args.given_gradient and info.path == B.DS_PATH_FUSED and args.workload == NCU_TRAFFIC["workload"] and not args.elems_per_lane
             and kernel_sources_digest() == NCU_TRAFFIC["sources_sha256"]):
         traffic = NCU_TRAFFIC["bytes_per_update"] * updates_per_step
     achieved = b_alg * updates_per_step / (kernel_ms * 1e-3) / 1e9
@@ -309,7 +318,7 @@ def main():
     # End to end through the host-buffer entry point: pinned host arrays in,
     # x and delta back out, every step.
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.given_gradient:
         hx = torch.zeros((w.n, ld), dtype=torch.float32).pin_memory()
         hd = torch.zeros((w.n, ld), dtype=torch.float32).pin_memory()
         ha = torch.from_numpy(a_h).pin_memory()
@@ -341,7 +350,8 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": w.describe(), "row_pitch": ld,
+                "config": {"workload": w.describe() + (" [gradient given: ds_step_g]" if args.given_gradient else ""),
+                           "row_pitch": ld,
                            "path": {B.DS_PATH_FUSED: "fused (persistent, TMA-staged)",
                                     B.DS_PATH_FUSED_LDG: "fused (direct loads)", B.DS_PATH_SPLIT: "split"}[info.path],
                            "elems_per_lane": info.elems_per_lane, "warps_per_chunk": info.warps_per_chunk,

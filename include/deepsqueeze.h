@@ -164,6 +164,18 @@ ds_status ds_init(ds_ctx **out, const ds_graph *graph, const float *W,
 ds_status ds_step(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
                   const ds_hparams *hp, uint64_t seed, uint64_t step, void *cuda_stream);
 
+/* The same iteration with the stochastic gradient SUPPLIED by the caller
+ * (Algorithm 1, gradient step: g_i = grad F_i(x_i; xi_i) from the caller's own
+ * training stack) instead of the synthetic objective:
+ *     v_i = x_i - gamma g_i + delta_i, compress, delta_i <- v_i - C[v_i],
+ *     x_i <- x_i - gamma g_i + eta sum_j (W_ij - I_ij) C[v_j].
+ *   g          device [n][ld], read only, 16-byte aligned, same pitch as x
+ *   seed,step  select the rounding stream of the b-bit compressor only
+ * Traffic: 20 + b/8 + 4/chunk bytes per node-element (one array less to read,
+ * no noise to generate). */
+ds_status ds_step_g(ds_ctx *ctx, float *x, float *delta, const float *g, const ds_hparams *hp,
+                    uint64_t seed, uint64_t step, void *cuda_stream);
+
 /* Same iteration for HOST buffers: copies x, delta, a, c (host, [n][ld]) into
  * the caller's device staging arrays, runs ds_step, and copies x and delta
  * back, all enqueued on `cuda_stream`; the caller synchronises the stream

@@ -303,6 +303,9 @@ void oracle_pack_codes(int bits, const uint32_t *q, int64_t first_elem,
  *   scales [n][scales_pitch]    one scale per (node, chunk)
  *   v_out, C_out (optional, [n][N])  the error-compensated variable and its
  *                               decoded compression, for the tests
+ *   g_given (optional, [n][ld])  the stochastic gradient itself (Algorithm 1,
+ *                               gradient step, computed by the caller); when not
+ *                               NULL, a, c, sigma and the noise are not used
  *   k_first                     global index of column 0 in the random streams:
  *                               0 for a whole problem; a multiple of the chunk
  *                               length when the arrays hold a window of columns
@@ -329,7 +332,7 @@ int oracle_step(int32_t n, int64_t N, int64_t ld,
                 uint64_t seed, uint64_t step,
                 uint32_t *codes, int64_t code_pitch,
                 float *scales, int64_t scales_pitch,
-                float *v_out, float *C_out, int64_t k_first)
+                float *v_out, float *C_out, int64_t k_first, const float *g_given)
 {
     if (chunk <= 0) chunk = N;
     int code_bits = (comp_kind == COMP_IDENTITY) ? 32
@@ -363,10 +366,15 @@ int oracle_step(int32_t n, int64_t N, int64_t ld,
             for (int64_t kk = 0; kk < m; ++kk) {
                 int64_t k = k0 + kk;
                 size_t at = (size_t)i * (size_t)ld + (size_t)k;
-                float z = oracle_noise_elem(noise_kind, seed, (uint32_t)i, step, k_first + k);
-                float d = x[at] - c[at];
-                float nz = sigma * z;
-                float g = fmaf(a[at], d, nz);
+                float g;
+                if (g_given) {
+                    g = g_given[at];         /* the caller's stochastic gradient */
+                } else {
+                    float z = oracle_noise_elem(noise_kind, seed, (uint32_t)i, step, k_first + k);
+                    float d = x[at] - c[at];
+                    float nz = sigma * z;
+                    g = fmaf(a[at], d, nz);
+                }
                 float hh = fmaf(-gamma, g, x[at]);
                 h[(size_t)i * (size_t)N + (size_t)k] = hh;
                 v[kk] = hh + delta[at];

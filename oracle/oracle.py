@@ -49,7 +49,7 @@ def lib():
             _f32p, _f32p, _f32p, _f32p,
             C.c_float, C.c_int, C.c_float, C.c_float,
             C.c_uint64, C.c_uint64,
-            _u32p, C.c_int64, _f32p, C.c_int64, _f32p, _f32p, C.c_int64]
+            _u32p, C.c_int64, _f32p, C.c_int64, _f32p, _f32p, C.c_int64, _f32p]
         L.oracle_step.restype = C.c_int
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = C.c_int
@@ -124,16 +124,17 @@ def code_bits(comp_kind: int, bits: int) -> int:
 def step(graph, comp_kind: int, bits: int, chunk: int, x: np.ndarray, delta: np.ndarray,
          a: np.ndarray, c: np.ndarray, N: int, sigma: float, noise_kind: int,
          gamma: float, eta: float, seed: int, step_index: int, want_vC: bool = False,
-         k_first: int = 0):
+         k_first: int = 0, g_given: np.ndarray | None = None):
     """One iteration in place on x, delta ([n][ld] float32, C-contiguous).
 
     Returns (codes [n][words] uint32, scales [n][M] float32, v, C) with v, C
     [n][N] float32 when want_vC, else None.  k_first > 0: the arrays hold the
     columns [k_first, k_first + N) of a longer problem (k_first a multiple of
     the chunk length); the random streams are indexed by the global column.
+    g_given: the stochastic gradient itself ([n][ld]); a, c, sigma, noise unused.
     """
     n, ld = x.shape
-    for arr in (x, delta, a, c):
+    for arr in (x, delta, a, c) + (() if g_given is None else (g_given,)):
         assert arr.dtype == np.float32 and arr.flags.c_contiguous and arr.shape == (n, ld)
     assert graph.n == n and N <= ld
     cb = code_bits(comp_kind, bits)
@@ -153,7 +154,8 @@ def step(graph, comp_kind: int, bits: int, chunk: int, x: np.ndarray, delta: np.
         _p(x, _f32p), _p(delta, _f32p), _p(a, _f32p), _p(c, _f32p),
         sigma, noise_kind, gamma, eta, seed, step_index,
         _p(codes, _u32p), words, _p(scales, _f32p), M,
-        _p(v, _f32p) if want_vC else None, _p(Cv, _f32p) if want_vC else None, k_first)
+        _p(v, _f32p) if want_vC else None, _p(Cv, _f32p) if want_vC else None, k_first,
+        None if g_given is None else _p(g_given, _f32p))
     if rc != 0:
         raise MemoryError("oracle_step could not allocate")
     return codes, scales, v, Cv

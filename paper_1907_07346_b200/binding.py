@@ -23,7 +23,7 @@ DS_COMP_IDENTITY, DS_COMP_SIGN1_L1, DS_COMP_UNIFORM_STOCH_MAXABS = 0, 1, 2
 DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 
-EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_host", "ds_codes", "ds_set_path",
+EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_g", "ds_step_host", "ds_codes", "ds_set_path",
            "ds_tune", "ds_get_info", "ds_sync", "ds_noise", "ds_node_scales_noalloc",
            "ds_destroy", "ds_strerror"]
 
@@ -69,6 +69,9 @@ def lib():
         L.ds_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ds_grad_params),
                               C.POINTER(ds_hparams), C.c_uint64, C.c_uint64, C.c_void_p]
         L.ds_step.restype = C.c_int
+        L.ds_step_g.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ds_hparams),
+                                C.c_uint64, C.c_uint64, C.c_void_p]
+        L.ds_step_g.restype = C.c_int
         L.ds_step_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                                    C.c_int32, C.POINTER(ds_hparams), C.c_uint64, C.c_uint64,
                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -180,6 +183,16 @@ class DeepSqueeze:
         s = torch.cuda.current_stream(self.device) if stream is None else stream
         _check(lib().ds_step(self.ctx, x.data_ptr(), delta.data_ptr(), C.byref(gp), C.byref(hp),
                              seed, step, C.c_void_p(s.cuda_stream)), "ds_step")
+
+    def ds_step_g(self, x, delta, g, gamma: float, eta: float, seed: int, step: int, stream=None):
+        """One iteration with the gradient supplied as a device tensor g[n][ld]."""
+        torch = self.torch
+        for t in (x, delta, g):
+            assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (self.n, self.ld)
+        hp = ds_hparams(gamma, eta)
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        _check(lib().ds_step_g(self.ctx, x.data_ptr(), delta.data_ptr(), g.data_ptr(), C.byref(hp),
+                               seed, step, C.c_void_p(s.cuda_stream)), "ds_step_g")
 
     def ds_step_host(self, x_h, delta_h, a_h, c_h, sigma, noise, gamma, eta, seed, step,
                      dev_x, dev_delta, dev_a, dev_c, stream=None):

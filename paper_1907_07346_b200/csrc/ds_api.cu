@@ -366,18 +366,19 @@ ds_status ds_codes(ds_ctx* ctx, const uint32_t** codes, int64_t* code_pitch_word
     return DS_OK;
 }
 
-ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const ds_hparams* hp,
-                  uint64_t seed, uint64_t step, void* cuda_stream) {
-    if (!ctx || !x || !delta || !gp || !hp || !gp->a || !gp->c) return DS_ERR_NULL;
-    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+// One iteration; `grad_kind` is a NOISE_* value for the synthetic gradient
+// (a, c given) or GRAD_GIVEN (a is the gradient itself, c unused).
+static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, const float* c,
+                          float sigma, int grad_kind, const ds_hparams* hp, uint64_t seed,
+                          uint64_t step, void* cuda_stream) {
     if (step >= ((uint64_t)1 << 56)) return DS_ERR_ARG;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
-                           reinterpret_cast<uintptr_t>(gp->a) | reinterpret_cast<uintptr_t>(gp->c);
+                           reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(c);
     if ((bits % 16) != 0) return DS_ERR_ALIGN;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     StepParams p;
-    p.x = x; p.delta = delta; p.a = gp->a; p.c = gp->c;
+    p.x = x; p.delta = delta; p.a = a; p.c = c;
     p.ld = ctx->ld; p.N = ctx->N; p.n = ctx->n; p.nnz = ctx->nnz;
     p.tile = ctx->sh.tile; p.tiles = ctx->sh.tiles;
     p.row_ptr = reinterpret_cast<const int32_t*>(ctx->base + ctx->ws.row_ptr);
@@ -390,7 +391,7 @@ ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp,
     p.scales_pitch = ctx->sh.scales_pitch;
     p.partials = reinterpret_cast<double*>(ctx->base + ctx->ws.partials);
     p.error_flag = reinterpret_cast<int*>(ctx->base + ctx->ws.error_flag);
-    p.sigma = gp->sigma;
+    p.sigma = sigma;
     p.neg_gamma = -hp->gamma;
     p.eta = hp->eta;
     p.rs = make_rng_step(seed, step);
@@ -398,7 +399,7 @@ ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp,
 
     auto shape_of = [&](const Plan& pl, int mode) {
         LaunchShape s;
-        s.code = ctx->sh.code; s.noise = gp->noise; s.elems_per_lane = pl.elems_per_lane;
+        s.code = ctx->sh.code; s.noise = grad_kind; s.elems_per_lane = pl.elems_per_lane;
         s.mode = mode; s.grid = pl.grid; s.block = pl.block; s.smem = pl.smem;
         return s;
     };
@@ -435,6 +436,19 @@ ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp,
         return DS_ERR_CUDA;
     }
     return DS_OK;
+}
+
+ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const ds_hparams* hp,
+                  uint64_t seed, uint64_t step, void* cuda_stream) {
+    if (!ctx || !x || !delta || !gp || !hp || !gp->a || !gp->c) return DS_ERR_NULL;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    return run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, gp->noise, hp, seed, step, cuda_stream);
+}
+
+ds_status ds_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, const ds_hparams* hp,
+                    uint64_t seed, uint64_t step, void* cuda_stream) {
+    if (!ctx || !x || !delta || !g || !hp) return DS_ERR_NULL;
+    return run_step(ctx, x, delta, g, nullptr, 0.0f, GRAD_GIVEN, hp, seed, step, cuda_stream);
 }
 
 ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const float* a_host,

@@ -118,10 +118,14 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
         if (FULL ? node_ok : (nv > 0)) {
             const float4 x4 = ld4(p.x + row + e0);
             const float4 d4 = ld4(p.delta + row + e0);
-            const float4 a4 = ld4(p.a + row + e0);
-            const float4 c4 = ld4(p.c + row + e0);
-            const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + e0));
-            local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
+            const float4 a4 = ld4(p.a + row + e0);      // the gradient itself when it is given
+            if constexpr (NOISE == GRAD_GIVEN) {
+                local_step4_given(x4, d4, a4, p.neg_gamma, &h[4 * r], &v[4 * r]);
+            } else {
+                const float4 c4 = ld4(p.c + row + e0);
+                const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + e0));
+                local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
+            }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 if (!FULL && j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
@@ -371,6 +375,7 @@ cudaError_t launch_code(const LaunchShape& sh, const StepParams& p, cudaStream_t
     DS_CASE(NOISE_NONE, 4) DS_CASE(NOISE_NONE, 8) DS_CASE(NOISE_NONE, 16)
     DS_CASE(NOISE_GAUSS, 4) DS_CASE(NOISE_GAUSS, 8) DS_CASE(NOISE_GAUSS, 16)
     DS_CASE(NOISE_T3, 4) DS_CASE(NOISE_T3, 8) DS_CASE(NOISE_T3, 16)
+    DS_CASE(GRAD_GIVEN, 4) DS_CASE(GRAD_GIVEN, 8) DS_CASE(GRAD_GIVEN, 16)
 #undef DS_CASE
     return cudaErrorInvalidValue;
 }

@@ -131,11 +131,12 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             const uint32_t bytes = (uint32_t)((len + 3) & ~3) * 4u;
             const size_t at = (size_t)node * (size_t)p.ld + (size_t)(col * p.tile) + (size_t)seg0;
             fence_proxy_async();      // earlier generic reads of the slot are ordered before the refill
-            mbar_expect_tx(bar, 4u * bytes);
+            constexpr uint32_t kArrays = (NOISE == GRAD_GIVEN) ? 3u : 4u;   // x, delta, g | x, delta, a, c
+            mbar_expect_tx(bar, kArrays * bytes);
             bulk_g2s(slot_addr + 0u * L.seg_bytes, p.x + at, bytes, bar);
             bulk_g2s(slot_addr + 1u * L.seg_bytes, p.delta + at, bytes, bar);
             bulk_g2s(slot_addr + 2u * L.seg_bytes, p.a + at, bytes, bar);
-            bulk_g2s(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar);
+            if constexpr (NOISE != GRAD_GIVEN) bulk_g2s(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar);
         }
         return true;
     };
@@ -182,9 +183,13 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     const float4 x4 = *reinterpret_cast<const float4*>(slot + 0 * SEG + e0);
                     const float4 d4 = *reinterpret_cast<const float4*>(slot + 1 * SEG + e0);
                     const float4 a4 = *reinterpret_cast<const float4*>(slot + 2 * SEG + e0);
-                    const float4 c4 = *reinterpret_cast<const float4*>(slot + 3 * SEG + e0);
-                    const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
-                    local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
+                    if constexpr (NOISE == GRAD_GIVEN) {
+                        local_step4_given(x4, d4, a4, p.neg_gamma, &h[4 * r], &v[4 * r]);
+                    } else {
+                        const float4 c4 = *reinterpret_cast<const float4*>(slot + 3 * SEG + e0);
+                        const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                        local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
+                    }
     #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         if (!FULL && j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
@@ -358,6 +363,7 @@ cudaError_t launch_tma_code(const LaunchShape& sh, const StepParams& p, cudaStre
     DS_TMA_CASE(NOISE_NONE, 4) DS_TMA_CASE(NOISE_NONE, 8) DS_TMA_CASE(NOISE_NONE, 16)
     DS_TMA_CASE(NOISE_GAUSS, 4) DS_TMA_CASE(NOISE_GAUSS, 8) DS_TMA_CASE(NOISE_GAUSS, 16)
     DS_TMA_CASE(NOISE_T3, 4) DS_TMA_CASE(NOISE_T3, 8) DS_TMA_CASE(NOISE_T3, 16)
+    DS_TMA_CASE(GRAD_GIVEN, 4) DS_TMA_CASE(GRAD_GIVEN, 8) DS_TMA_CASE(GRAD_GIVEN, 16)
 #undef DS_TMA_CASE
     return cudaErrorInvalidValue;
 }

@@ -78,11 +78,15 @@ __device__ __forceinline__ void wide_column(const StepParams& p, const WideSmemL
             if (nv > 0) {
                 const float4 x4 = ld4(p.x + row + e0);
                 const float4 d4 = ld4(p.delta + row + e0);
-                const float4 a4 = ld4(p.a + row + e0);
-                const float4 c4 = ld4(p.c + row + e0);
-                const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + e0));
+                const float4 a4 = ld4(p.a + row + e0);      // the gradient itself when it is given
                 float h[4];
-                local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, h, &v[4 * r]);
+                if constexpr (NOISE == GRAD_GIVEN) {
+                    local_step4_given(x4, d4, a4, p.neg_gamma, h, &v[4 * r]);
+                } else {
+                    const float4 c4 = ld4(p.c + row + e0);
+                    const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + e0));
+                    local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, h, &v[4 * r]);
+                }
                 // park x - gamma g in x (read back by this same thread in sweep 2)
                 if (FULL || nv == 4) {
                     *reinterpret_cast<float4*>(p.x + row + e0) = make_float4(h[0], h[1], h[2], h[3]);
@@ -303,6 +307,7 @@ cudaError_t launch_wide_code(const LaunchShape& sh, const StepParams& p, cudaStr
     DS_WIDE_CASE(NOISE_NONE, 4) DS_WIDE_CASE(NOISE_NONE, 8) DS_WIDE_CASE(NOISE_NONE, 16)
     DS_WIDE_CASE(NOISE_GAUSS, 4) DS_WIDE_CASE(NOISE_GAUSS, 8) DS_WIDE_CASE(NOISE_GAUSS, 16)
     DS_WIDE_CASE(NOISE_T3, 4) DS_WIDE_CASE(NOISE_T3, 8) DS_WIDE_CASE(NOISE_T3, 16)
+    DS_WIDE_CASE(GRAD_GIVEN, 4) DS_WIDE_CASE(GRAD_GIVEN, 8) DS_WIDE_CASE(GRAD_GIVEN, 16)
 #undef DS_WIDE_CASE
     return cudaErrorInvalidValue;
 }

@@ -253,3 +253,45 @@ def test_host_buffer_entry_point(env):
     assert row_rel_err(host[0].numpy()[:, :N], x[:, :N]) <= TOL_STEP
     assert row_rel_err(host[1].numpy()[:, :N], d[:, :N]) <= TOL_STEP
     ds.close()
+
+
+# ------------------------------------------- gradient supplied by the caller
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("case", [("ring16", I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, 512 * 5 + 40),
+                                  ("torus4x8", I.COMP_UNIFORM_STOCH_MAXABS, 2, 256, 256 * 6 + 3),
+                                  ("exp64", I.COMP_SIGN1_L1, 1, 1024, 1024 * 2 + 130),
+                                  ("ring8", I.COMP_SIGN1_L1, 1, 4096, 4096 * 2 + 74),
+                                  ("ring4", I.COMP_SIGN1_L1, 1, 0, 5000),
+                                  ("ring8", I.COMP_UNIFORM_STOCH_MAXABS, 8, 96, 96 * 5 + 1)])
+def test_given_gradient_steps(env, path, case):
+    """ds_step_g against the oracle fed the same gradients, 3 free-running steps."""
+    torch, orc, B = env
+    gname, kind, bits, chunk, N = case
+    g = {"ring4": I.ring(4), "ring8": I.ring(8), "ring16": I.ring(16), "torus4x8": I.torus(4, 8),
+         "exp64": I.exponential(64)}[gname]
+    ld = I.round_up(N, 4)
+    x, d, _, _ = make_state(g, N, ld, 31)
+    rng = np.random.default_rng(77)
+    ds = B.DeepSqueeze(g, N, ld, kind, bits, chunk)
+    try:
+        ds.ds_set_path(path)
+    except B.DsError:
+        ds.close()
+        pytest.skip("shape not available on this path")
+    dx, dd = torch.from_numpy(x.copy()).cuda(), torch.from_numpy(d.copy()).cuda()
+    zeros = np.zeros_like(x)
+    for t in range(3):
+        grad = np.zeros_like(x)
+        grad[:, :N] = rng.standard_normal((g.n, N)).astype(np.float32)
+        grad[:, N:] = 9.0
+        codes_ref, scales_ref, _, _ = orc.step(g, kind, bits, chunk, x, d, zeros, zeros, N, 0.0,
+                                               I.NOISE_NONE, 0.05, 0.5, 5, t, g_given=grad)
+        ds.ds_step_g(dx, dd, torch.from_numpy(grad).cuda(), 0.05, 0.5, 5, t)
+        ds.ds_sync()
+        codes, scales = ds.codes_to_host()
+        assert np.array_equal(codes, codes_ref)
+        assert row_rel_err(scales, scales_ref) <= TOL_STEP
+        gx, gd = dx.cpu().numpy(), dd.cpu().numpy()
+        assert row_rel_err(gx[:, :N], x[:, :N]) <= TOL_STEP and row_rel_err(gd[:, :N], d[:, :N]) <= TOL_STEP
+        assert np.array_equal(gx[:, N:], x[:, N:]) and np.array_equal(gd[:, N:], d[:, N:])
+    ds.close()

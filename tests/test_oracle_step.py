@@ -298,3 +298,40 @@ def test_column_window_equals_slice_of_whole_problem(comp):
         assert np.array_equal(sw, scales[:, k_first // chunk:k_first // chunk + sw.shape[1]])
         w0 = k_first * comp[1] // 32
         assert np.array_equal(cw, codes[:, w0:w0 + cw.shape[1]])
+
+
+@pytest.mark.parametrize("comp", [(I.COMP_SIGN1_L1, 1, 32), (I.COMP_UNIFORM_STOCH_MAXABS, 4, 64),
+                                  (I.COMP_IDENTITY, 32, 0)])
+def test_given_gradient_reproduces_synthetic_step(comp):
+    """Algorithm 1 takes any stochastic gradient.  Feeding the iteration the
+    gradient of the synthetic objective, evaluated outside (a (x - c) + sigma z
+    in binary32, the product-sum with one rounding), must reproduce the
+    synthetic step bit for bit; and the identities hold for an arbitrary g."""
+    kind, bits, chunk = comp
+    g = I.torus(3, 4)
+    N = 150
+    x, d, a, c = make_problem(g, N, 23, pad=2)
+    x2, d2 = x.copy(), d.copy()
+    sigma, gamma, eta, seed, t = 0.1, 0.05, 0.5, 9, 4
+    z = np.zeros_like(x)
+    for i in range(g.n):
+        z[i, :N] = orc.noise_row(I.NOISE_GAUSS, seed, i, t, 0, N)
+    dd = (x - c).astype(np.float32)
+    nz = (np.float32(sigma) * z).astype(np.float32)
+    grad = (a.astype(np.float64) * dd.astype(np.float64) + nz.astype(np.float64)).astype(np.float32)
+    ref = orc.step(g, kind, bits, chunk, x, d, a, c, N, sigma, I.NOISE_GAUSS, gamma, eta, seed, t)
+    got = orc.step(g, kind, bits, chunk, x2, d2, a, c, N, 0.0, I.NOISE_NONE, gamma, eta, seed, t,
+                   g_given=grad)
+    assert np.array_equal(x, x2) and np.array_equal(d, d2)
+    assert np.array_equal(ref[0], got[0]) and np.array_equal(ref[1], got[1])
+    # arbitrary gradient: compression identity and mean preservation
+    rng = np.random.default_rng(3)
+    x3, d3, _, _ = make_problem(g, N, 24)
+    x0, d0 = x3.copy(), d3.copy()
+    grad = rng.standard_normal(x3.shape).astype(np.float32)
+    _, _, v, Cv = orc.step(g, kind, bits, chunk, x3, d3, x3 * 0, x3 * 0, N, 0.0, I.NOISE_NONE, gamma, eta,
+                           seed, t, want_vC=True, g_given=grad)
+    H = x0.astype(np.float64) - gamma * grad
+    assert np.allclose(v, H + d0, atol=2e-6, rtol=0)
+    assert np.abs(Cv.astype(np.float64) + d3 - v).max() <= 2.4e-7 * max(1.0, np.abs(v).max())
+    assert np.allclose(x3.astype(np.float64).mean(0), H.mean(0), atol=3e-6, rtol=0)
