@@ -217,6 +217,13 @@ ds_status ds_get_info(const ds_ctx *ctx, ds_info *info);
  * the step early instead of hanging the device. */
 ds_status ds_sync(ds_ctx *ctx, void *cuda_stream);
 
+/* Failure-reporting self-test: enqueues a one-warp kernel that waits, with a
+ * small fixed budget, on a completion that never comes, gives up and raises the
+ * context's error flag exactly as the fused kernel does when a staged copy does
+ * not arrive.  The next ds_sync must return DS_ERR_TIMEOUT (and clear the flag).
+ * Nothing hangs and nothing faults; x and delta are not touched. */
+ds_status ds_selftest_timeout(ds_ctx *ctx, void *cuda_stream);
+
 /* Diagnostics: write the random streams the kernels draw from, one value per
  * element, out[node][k] for k < N (device, [n][ld_out]).  which = 0: unit
  * gradient noise z of kind `noise`; which = 1: the rounding uniforms in

@@ -24,7 +24,7 @@ DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 
 EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_g", "ds_step_host", "ds_codes", "ds_set_path",
-           "ds_tune", "ds_get_info", "ds_sync", "ds_noise", "ds_node_scales_noalloc",
+           "ds_tune", "ds_get_info", "ds_sync", "ds_selftest_timeout", "ds_noise", "ds_node_scales_noalloc",
            "ds_destroy", "ds_strerror"]
 
 
@@ -87,6 +87,8 @@ def lib():
         L.ds_get_info.restype = C.c_int
         L.ds_sync.argtypes = [C.c_void_p, C.c_void_p]
         L.ds_sync.restype = C.c_int
+        L.ds_selftest_timeout.argtypes = [C.c_void_p, C.c_void_p]
+        L.ds_selftest_timeout.restype = C.c_int
         L.ds_noise.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
                                C.c_uint64, C.c_uint64, C.c_void_p]
         L.ds_noise.restype = C.c_int
@@ -210,6 +212,10 @@ class DeepSqueeze:
         """Synchronise the stream and raise if a kernel gave up on a bounded wait."""
         s = self.torch.cuda.current_stream(self.device) if stream is None else stream
         _check(lib().ds_sync(self.ctx, C.c_void_p(s.cuda_stream)), "ds_sync")
+
+    def ds_selftest_timeout(self, stream=None):
+        s = self.torch.cuda.current_stream(self.device) if stream is None else stream
+        _check(lib().ds_selftest_timeout(self.ctx, C.c_void_p(s.cuda_stream)), "ds_selftest_timeout")
 
     def ds_codes(self):
         """(codes_ptr, code_pitch_words, scales_ptr, scales_pitch) of the last step."""

@@ -488,6 +488,14 @@ ds_status ds_sync(ds_ctx* ctx, void* cuda_stream) {
     return DS_OK;
 }
 
+ds_status ds_selftest_timeout(ds_ctx* ctx, void* cuda_stream) {
+    if (!ctx) return DS_ERR_NULL;
+    const cudaError_t e = launch_wait_selftest(reinterpret_cast<int*>(ctx->base + ctx->ws.error_flag),
+                                               static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+    return DS_OK;
+}
+
 ds_status ds_noise(float* out, int32_t n, int64_t N, int64_t ld_out, int32_t which, int32_t noise,
                    uint64_t seed, uint64_t step, void* cuda_stream) {
     if (!out) return DS_ERR_NULL;

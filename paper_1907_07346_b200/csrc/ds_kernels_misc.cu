@@ -1,6 +1,6 @@
 // Mix kernel of the two-kernel path, the per-node scale finaliser and the
 // random-stream diagnostic kernel.
-#include "ds_column_kernel.cuh"
+#include "ds_fused_tma_kernel.cuh"
 
 namespace ds {
 
@@ -146,6 +146,27 @@ cudaError_t launch_noise_kernel(float* out, int32_t n, int64_t N, int64_t ld, in
     int64_t bx = (nf4 + 255) / 256;
     if (bx > 148 * 32) bx = 148 * 32;
     ds_noise_kernel<<<dim3((unsigned)bx, (unsigned)n), 256, 0, stream>>>(out, n, N, ld, which, noise, rs);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Self-test of the bounded wait: one warp waits, for at most 20 ms, on an
+// mbarrier that nothing ever completes, gives up, and raises the error flag --
+// the same give-up path the fused kernel takes when a bulk copy does not
+// arrive.  The kernel always terminates.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) ds_wait_selftest_kernel(int* error_flag) {
+    __shared__ __align__(8) unsigned long long bar_storage;
+    const uint32_t bar = smem_u32(&bar_storage);
+    if (threadIdx.x == 0) mbar_init(bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    const bool done = mbar_wait_bounded(bar, 0u, 20000000ull);      // 20 ms
+    if (!done && threadIdx.x == 0) *error_flag = 1;
+}
+
+cudaError_t launch_wait_selftest(int* error_flag, cudaStream_t stream) {
+    ds_wait_selftest_kernel<<<1, 32, 0, stream>>>(error_flag);
     return cudaGetLastError();
 }
 

@@ -295,3 +295,42 @@ def test_given_gradient_steps(env, path, case):
         assert row_rel_err(gx[:, :N], x[:, :N]) <= TOL_STEP and row_rel_err(gd[:, :N], d[:, :N]) <= TOL_STEP
         assert np.array_equal(gx[:, N:], x[:, N:]) and np.array_equal(gd[:, N:], d[:, N:])
     ds.close()
+
+
+# --------------------------------------------------- failure reporting, odd graphs
+def test_bounded_wait_reports_timeout_and_context_stays_usable(env):
+    """A wait that runs out is reported by ds_sync as DS_ERR_TIMEOUT (once), no
+    hang, no fault, and the context keeps working afterwards."""
+    torch, orc, B = env
+    g = I.ring(4)
+    N, ld = 512 * 2, 512 * 2
+    ds = B.DeepSqueeze(g, N, ld, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512)
+    ds.ds_sync()
+    ds.ds_selftest_timeout()
+    with pytest.raises(B.DsError) as err:
+        ds.ds_sync()
+    assert err.value.status == B.DS_ERR_TIMEOUT
+    ds.ds_sync()                                   # the flag was cleared
+    x, d, a, c = make_state(g, N, ld, 3)
+    dev = [torch.from_numpy(t.copy()).cuda() for t in (x, d, a, c)]
+    orc.step(g, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, x, d, a, c, N, 0.1, I.NOISE_GAUSS, 0.05, 0.5, 1, 0)
+    ds.ds_step(dev[0], dev[1], dev[2], dev[3], 0.1, I.NOISE_GAUSS, 0.05, 0.5, 1, 0)
+    ds.ds_sync()
+    assert row_rel_err(dev[0].cpu().numpy(), x) <= TOL_STEP
+    ds.close()
+
+
+def _complete_graph(n):
+    rp = np.arange(0, n * n + 1, n, dtype=np.int32)
+    ci = np.tile(np.arange(n, dtype=np.int32), n)
+    return I.Graph(n, rp, ci, np.full(n * n, 1.0 / n, np.float32), f"complete{n}")
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("g", [_complete_graph(1), _complete_graph(2), I.ring(3), I.ring(40), _complete_graph(7)],
+                         ids=["single", "pair", "ring3", "ring40", "complete7"])
+def test_unusual_graphs(env, path, g):
+    """One node alone (W = [1], the mixing term vanishes), a pair, a node count
+    that is not a multiple of the block's batch, a dense neighbourhood."""
+    run_case(env, g, 512 * 2 + 17, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_GAUSS, path)
+    run_case(env, g, 1024 + 9, I.COMP_SIGN1_L1, 1, 1024, I.NOISE_GAUSS, path)
