@@ -71,11 +71,19 @@ typedef struct {
  *   DS_COMP_UNIFORM_STOCH_MAXABS b in {1,2,4,8} bits: 2^b levels evenly spaced on
  *                                [-s, s], s = max |v| over the chunk, stochastic rounding
  *                                with a Philox4x32-10 stream; unbiased.
+ *   DS_COMP_UNIFORM_NEAREST_L2   the paper's own "bit compression" (Section 5): b in {2,4} bits,
+ *                                each element rounded to the NEAREST of 2^b levels spanning
+ *                                [-max|v|, max|v|]; the scalar sent with the chunk is the
+ *                                Euclidean norm ||v||_2, and the receiver rescales what it
+ *                                decodes to that norm: C = level[code] * ||v||_2 / ||level[code]||_2.
+ *                                Deterministic and biased -- what error compensation is for.
+ *                                chunk must be in 32..512 (one chunk = one "tensor").
  * chunk: elements per scale, a multiple of 32; 0 = one scale per node. */
 typedef enum {
     DS_COMP_IDENTITY = 0,
     DS_COMP_SIGN1_L1 = 1,
-    DS_COMP_UNIFORM_STOCH_MAXABS = 2
+    DS_COMP_UNIFORM_STOCH_MAXABS = 2,
+    DS_COMP_UNIFORM_NEAREST_L2 = 3
 } ds_comp_kind;
 
 typedef struct {

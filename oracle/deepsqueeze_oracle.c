@@ -203,7 +203,8 @@ float oracle_rnd24_elem(uint64_t seed, uint32_t node, uint64_t step, int64_t k)
 /* Compressors C_omega (Algorithm 1, compression step; Section 5,       */
 /* "Compression": b bits per element plus one scalar per tensor).       */
 /* ------------------------------------------------------------------ */
-enum { COMP_IDENTITY = 0, COMP_SIGN1_L1 = 1, COMP_UNIFORM_STOCH_MAXABS = 2 };
+enum { COMP_IDENTITY = 0, COMP_SIGN1_L1 = 1, COMP_UNIFORM_STOCH_MAXABS = 2,
+       COMP_UNIFORM_NEAREST_L2 = 3 };
 
 /* Reconstruction level q of the b-bit grid: 2^b points evenly spaced on
  * [-1, 1] including both ends. */
@@ -223,7 +224,16 @@ float oracle_level(int bits, int q)
  *              code = clamp(floor(u + r_k), 0, L), C_k = s * level[code].
  *              NaN elements code to 0.
  *   IDENTITY : C_k = v_k, the "code" is the bit pattern of v_k.
- * q_out receives one code per element (unpacked).
+ *   NEAREST_L2 : the paper's "bit compression" (Section 5, "Compression"): b bits
+ *              per element and the Euclidean norm of the tensor, the receiver
+ *              rescaling what it decodes to that norm.  Grid as above with
+ *              g = max|v_k|: code = clamp(floor(fma(v_k/g, L/2, L/2) + 1/2), 0, L)
+ *              (nearest level), l_k = level[code]; the scalar sent is
+ *              nrm = sqrt(sum v_k^2), the receiver forms lnorm = sqrt(sum l_k^2)
+ *              (both sums in binary64, rounded to binary32) and
+ *              C_k = (nrm / lnorm) * l_k.  g = 0 or not finite, or a norm that is
+ *              not finite: nrm = 0 is sent and C = 0 * l_k.
+ * q_out receives one code per element (unpacked); *scale_out is what is sent.
  */
 void oracle_compress_chunk(int kind, int bits, const float *v, int64_t m,
                            const float *r, float *scale_out,
@@ -247,6 +257,36 @@ void oracle_compress_chunk(int kind, int bits, const float *v, int64_t m,
             C_out[k] = bit ? s : -s;
         }
         *scale_out = s;
+        return;
+    }
+    if (kind == COMP_UNIFORM_NEAREST_L2) {
+        int L = (1 << bits) - 1;
+        float g = 0.0f;
+        for (int64_t k = 0; k < m; ++k) g = fmaxf(g, fabsf(v[k]));
+        int dead = (g == 0.0f || !isfinite(g));
+        float hl = 0.5f * (float)L;
+        double sv2 = 0.0, sl2 = 0.0;
+        for (int64_t k = 0; k < m; ++k) {
+            int q = 0;
+            if (!dead) {
+                float y = v[k] / g;
+                float u = fmaf(y, hl, hl);
+                float t = floorf(u + 0.5f);
+                if (t >= 1.0f) q = (t >= (float)L) ? L : (int)t;
+            }
+            q_out[k] = (uint32_t)q;
+            float l = oracle_level(bits, q);
+            C_out[k] = l;                          /* unit reconstruction for now */
+            sv2 += (double)v[k] * (double)v[k];
+            sl2 += (double)l * (double)l;
+        }
+        float nrm = dead ? 0.0f : (float)sqrt(sv2);
+        float lnorm = (float)sqrt(sl2);
+        float ratio = 0.0f;
+        if (!dead && lnorm != 0.0f && isfinite(nrm)) ratio = nrm / lnorm;
+        if (!isfinite(nrm)) nrm = 0.0f;
+        for (int64_t k = 0; k < m; ++k) C_out[k] = ratio * C_out[k];
+        *scale_out = nrm;
         return;
     }
     /* COMP_UNIFORM_STOCH_MAXABS */

@@ -19,7 +19,7 @@ DS_OK = 0
  DS_ERR_NO_SELF_LOOP, DS_ERR_ALIGN, DS_ERR_WORKSPACE, DS_ERR_UNSUPPORTED, DS_ERR_CUDA,
  DS_ERR_TIMEOUT) = range(1, 12)
 
-DS_COMP_IDENTITY, DS_COMP_SIGN1_L1, DS_COMP_UNIFORM_STOCH_MAXABS = 0, 1, 2
+DS_COMP_IDENTITY, DS_COMP_SIGN1_L1, DS_COMP_UNIFORM_STOCH_MAXABS, DS_COMP_UNIFORM_NEAREST_L2 = 0, 1, 2, 3
 DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 

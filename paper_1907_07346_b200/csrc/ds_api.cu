@@ -33,7 +33,7 @@ struct Shape {
 };
 
 struct WsLayout {
-    size_t codes, scales, partials, row_ptr, col_idx, wprime, lut, error_flag, total;
+    size_t codes, scales, dscales, partials, row_ptr, col_idx, wprime, lut, error_flag, total;
 };
 
 bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
@@ -50,6 +50,13 @@ bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
             else if (comp->bits == 4) sh->code = CODE_U4;
             else if (comp->bits == 8) sh->code = CODE_U8;
             else return false;
+            break;
+        case DS_COMP_UNIFORM_NEAREST_L2:
+            // the paper's own settings (2 and 4 bits); one warp codes a chunk, so chunk <= 512
+            if (comp->bits == 2) sh->code = CODE_N2;
+            else if (comp->bits == 4) sh->code = CODE_N4;
+            else return false;
+            if (comp->chunk < 32 || comp->chunk > 512) return false;
             break;
         default: return false;
     }
@@ -72,6 +79,9 @@ WsLayout make_ws(int32_t n, int32_t nnz, const Shape& sh) {
     size_t off = 0;
     w.codes = off;    off = align_up(off + (size_t)n * (size_t)sh.code_pitch * 4, kAlign);
     w.scales = off;   off = align_up(off + (size_t)n * (size_t)sh.scales_pitch * 4, kAlign);
+    const bool norm = (sh.code == CODE_N2 || sh.code == CODE_N4);
+    w.dscales = norm ? off : w.scales;      // decode factors only differ from the sent scalars for norm-matched codes
+    if (norm) off = align_up(off + (size_t)n * (size_t)sh.scales_pitch * 4, kAlign);
     w.partials = off; off = align_up(off + (sh.per_node ? (size_t)n * (size_t)sh.tiles * 8 : 0), kAlign);
     w.row_ptr = off;  off = align_up(off + (size_t)(n + 1) * 4, kAlign);
     w.col_idx = off;  off = align_up(off + (size_t)nnz * 4, kAlign);
@@ -103,6 +113,7 @@ Plan plan_column(int mode, const Shape& sh, int32_t n, int32_t nnz, int force_e 
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
     if (G > 32) return pl;
+    if ((sh.code == CODE_N2 || sh.code == CODE_N4) && G != 1) return pl;
     int npb;
     if (mode == MODE_FUSED) {
         if (sh.code == CODE_ID32) return pl;
@@ -129,6 +140,7 @@ Plan plan_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int force_e 
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
     if (sh.code == CODE_ID32 || (int64_t)n * G > 32 || num_sms < 1) return pl;
+    if ((sh.code == CODE_N2 || sh.code == CODE_N4) && G != 1) return pl;
     // every warp of a group owns a whole E*32-element segment
     if ((int64_t)G * E * 32 < sh.tile) return pl;
     pl.nodes_per_block = n;
@@ -148,7 +160,7 @@ Plan plan_wide(const Shape& sh, int32_t n, int32_t nnz, int force_e = 0) {
     pick_lane_shape(sh.tile, force_e, &E, &G);
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
-    if (sh.code == CODE_ID32 || G > 16) return pl;
+    if (sh.code == CODE_ID32 || sh.code == CODE_N2 || sh.code == CODE_N4 || G > 16) return pl;
     const int npb = std::max(1, std::min<int>(n, 16 / G));
     pl.nodes_per_block = npb;
     pl.block = dim3((unsigned)(npb * G * 32));
@@ -208,7 +220,7 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     if (n < 1 || N < 1 || N >= ((int64_t)1 << 31) || graph->n != n || ld < N) return DS_ERR_ARG;
     if ((ld % 4) != 0) return DS_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(workspace) % kAlign) != 0) return DS_ERR_ALIGN;
-    if (comp->kind < DS_COMP_IDENTITY || comp->kind > DS_COMP_UNIFORM_STOCH_MAXABS) return DS_ERR_ARG;
+    if (comp->kind < DS_COMP_IDENTITY || comp->kind > DS_COMP_UNIFORM_NEAREST_L2) return DS_ERR_ARG;
     if (comp->chunk < 0 || (comp->chunk % 32) != 0) return DS_ERR_ARG;
     Shape sh;
     if (!make_shape(n, N, comp, &sh)) return DS_ERR_UNSUPPORTED;
@@ -294,7 +306,7 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.wprime, wprime.data(), (size_t)nnz * 4, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.lut, lut, sizeof(lut), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.codes, 0, ws.scales - ws.codes);
-    if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.scales, 0, ws.partials - ws.scales);
+    if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.scales, 0, ws.partials - ws.scales);   // scales and decode factors
     if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.error_flag, 0, 4);
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
@@ -389,6 +401,7 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
     p.code_pitch = ctx->sh.code_pitch;
     p.scales = reinterpret_cast<float*>(ctx->base + ctx->ws.scales);
     p.scales_pitch = ctx->sh.scales_pitch;
+    p.dscales = reinterpret_cast<float*>(ctx->base + ctx->ws.dscales);
     p.partials = reinterpret_cast<double*>(ctx->base + ctx->ws.partials);
     p.error_flag = reinterpret_cast<int*>(ctx->base + ctx->ws.error_flag);
     p.sigma = sigma;

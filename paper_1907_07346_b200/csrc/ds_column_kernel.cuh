@@ -60,9 +60,10 @@ template <int CODE>
 struct CodeTraits {
     static constexpr bool kSign = (CODE == CODE_SIGN);
     static constexpr bool kIdentity = (CODE == CODE_ID32);
+    static constexpr bool kNorm = (CODE == CODE_N2 || CODE == CODE_N4);
     static constexpr int kBits = (CODE == CODE_SIGN || CODE == CODE_U1) ? 1
-                               : (CODE == CODE_U2) ? 2
-                               : (CODE == CODE_U4) ? 4
+                               : (CODE == CODE_U2 || CODE == CODE_N2) ? 2
+                               : (CODE == CODE_U4 || CODE == CODE_N4) ? 4
                                : (CODE == CODE_U8) ? 8 : 32;
     static constexpr bool kLut = !(kSign || kIdentity);
     static constexpr bool kTable = kLut && kBits <= 4;   // per-node decode table in shared memory
@@ -75,6 +76,61 @@ __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+
+// Norm-matched b-bit compression of one chunk held by ONE warp (Section 5,
+// "Compression": b bits per element plus the Euclidean norm of the tensor; the
+// receiver rescales what it decodes to that norm).
+//   m = max |v| spans the grid; code = clamp(floor(fma(v/m, L/2, L/2) + 1/2), 0, L)
+//   (round to nearest level); l_k = level[code_k];
+//   nrm = sqrt(sum v_k^2), lnorm = sqrt(sum l_k^2) (binary64 sums, rounded to binary32);
+//   r = nrm / lnorm;  C_k = r * l_k.
+// A lane holds E elements, element 4*(32*r + lane) + j of the chunk at index
+// 4*r + j; only the first valid_len elements of the chunk count.  On return
+// q[] holds the codes, cv[] the C values, nrm the scalar to send and r the
+// decode factor.  m = 0 or not finite: codes 0, nrm = r = 0.
+template <int CODE, int E, bool FULL>
+__device__ __forceinline__ void norm_compress(const float* v, int valid_len, float m, const float* lut,
+                                              int lane, uint32_t* q, float* cv, float& nrm, float& r) {
+    constexpr int kBits = (CODE == CODE_N2) ? 2 : 4;
+    constexpr int kLi = (1 << kBits) - 1;
+    constexpr float kHalfL = 0.5f * (float)kLi;
+    const bool dead = (m == 0.0f) || !(m <= 3.402823466e+38f);
+    const bool fast = !dead && m >= 0x1p-60f && m <= 0x1p+60f;
+    const float inv = fast ? __fdiv_rn(1.0f, m) : 0.0f;
+    double sv2 = 0.0, sl2 = 0.0;
+#pragma unroll
+    for (int t = 0; t < E; ++t) {
+        const int k = 4 * (32 * (t >> 2) + lane) + (t & 3);
+        const bool ok = FULL || k < valid_len;
+        float y;
+        if (fast) {
+            const float q0 = __fmul_rn(v[t], inv);
+            const float rem = __fmaf_rn(-q0, m, v[t]);
+            y = __fmaf_rn(rem, inv, q0);
+        } else {
+            y = dead ? 0.0f : __fdiv_rn(v[t], m);
+        }
+        const float u = __fmaf_rn(y, kHalfL, kHalfL);
+        const uint32_t code = dead ? 0u : (uint32_t)min(max(__float2int_rd(__fadd_rn(u, 0.5f)), 0), kLi);
+        q[t] = code;
+        cv[t] = lut[code];
+        if (ok) {
+            sv2 += (double)v[t] * (double)v[t];
+            sl2 += (double)cv[t] * (double)cv[t];
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        sv2 += __shfl_xor_sync(0xffffffffu, sv2, o);
+        sl2 += __shfl_xor_sync(0xffffffffu, sl2, o);
+    }
+    nrm = dead ? 0.0f : (float)sqrt(sv2);
+    const float lnorm = (float)sqrt(sl2);
+    r = (dead || lnorm == 0.0f || !(nrm <= 3.402823466e+38f)) ? 0.0f : __fdiv_rn(nrm, lnorm);
+    if (!(nrm <= 3.402823466e+38f)) nrm = 0.0f;
+#pragma unroll
+    for (int t = 0; t < E; ++t) cv[t] = __fmul_rn(r, cv[t]);
 }
 
 __device__ __forceinline__ float4 ld4(const float* p) {
@@ -185,6 +241,17 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
     const size_t code_row = (size_t)node * (size_t)p.code_pitch
                           + (size_t)((k0 * T::kBits) >> 5);
 
+    // norm-matched codes (one warp per chunk only): code the whole chunk first;
+    // s becomes the norm that is sent, dscale the factor the receiver applies
+    uint32_t qn[T::kNorm ? E : 1];
+    float cvn[T::kNorm ? E : 1];
+    float dscale = s;
+    if constexpr (T::kNorm) {
+        float nrm;
+        norm_compress<CODE, E, FULL>(v, node_ok ? m_len : 0, s, lut, lane, qn, cvn, nrm, dscale);
+        s = nrm;
+    }
+
     // ---------------- phase B: compress, residual, pack ------------------
     constexpr float kL = (float)((1u << (T::kBits & 15)) - 1u);
     constexpr float kHalfL = 0.5f * kL;
@@ -206,7 +273,13 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
         } else {
             if (nv > 0) {
                 float dn[4];
-                if constexpr (T::kSign) {
+                if constexpr (T::kNorm) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        dn[j] = __fadd_rn(v[4 * r + j], -cvn[4 * r + j]);
+                        if (FULL || j < nv) piece |= qn[4 * r + j] << (T::kBits * j);
+                    }
+                } else if constexpr (T::kSign) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const uint32_t bit = (v[4 * r + j] >= 0.0f) ? 1u : 0u;
@@ -254,15 +327,17 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
         }
     }
     if constexpr (!T::kIdentity) {
-        if (!p.prescaled && node_ok && wg == 0 && lane == 0)
+        if (!p.prescaled && node_ok && wg == 0 && lane == 0) {
             p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+            if constexpr (T::kNorm) p.dscales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = dscale;
+        }
     }
 
     if constexpr (MODE == MODE_FUSED) {
-        if (wg == 0 && lane == 0) scale_sm[grp] = s;
+        if (wg == 0 && lane == 0) scale_sm[grp] = dscale;
         float* table_sm = reinterpret_cast<float*>(smem + L.table_off) + buf * p.nodes_per_block * 16;
         if constexpr (T::kTable) {
-            if (wg == 0 && lane < (1 << T::kBits)) table_sm[grp * 16 + lane] = __fmul_rn(s, lut[lane]);
+            if (wg == 0 && lane < (1 << T::kBits)) table_sm[grp * 16 + lane] = __fmul_rn(dscale, lut[lane]);
         }
         __syncthreads();    // codes and scales of all nodes of this tile are in shared memory
 

@@ -251,6 +251,16 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             const float inv_s = fast ? __fdiv_rn(1.0f, s) : 0.0f;
             const size_t code_row = (size_t)node * (size_t)p.code_pitch + (size_t)(((k0 + seg0) * T::kBits) >> 5);
             float* cval_mine = cval + (size_t)node * p.tile + seg0;
+            // norm-matched codes: the whole chunk is coded first (two more warp
+            // reductions), s becomes the norm that is sent, dscale the decode factor
+            uint32_t qn[T::kNorm ? E : 1];
+            float cvn[T::kNorm ? E : 1];
+            float dscale = s;
+            if constexpr (T::kNorm) {
+                float nrm;
+                norm_compress<CODE, E, FULL>(v, live_len, s, lut, lane, qn, cvn, nrm, dscale);
+                s = nrm;
+            }
 
             // ---- phase B: compress, residual, pack -----------------------------
     #pragma unroll
@@ -261,7 +271,13 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 uint32_t piece = 0u;
                 if (nv > 0) {
                     float dn[4], cv[4];
-                    if constexpr (T::kSign) {
+                    if constexpr (T::kNorm) {
+    #pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            cv[j] = cvn[4 * r + j];
+                            if (FULL || j < nv) piece |= qn[4 * r + j] << (T::kBits * j);
+                        }
+                    } else if constexpr (T::kSign) {
     #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const uint32_t bit = (v[4 * r + j] >= 0.0f) ? 1u : 0u;
@@ -304,7 +320,10 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     p.codes[code_row + f / T::kLanesPerWord] = word;
             }
             if (!p.prescaled && alive && wg == 0 && lane == 0)
+            {
                 p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+                if constexpr (T::kNorm) p.dscales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = dscale;
+            }
 
             __syncthreads();       // C[v] of every node of this tile is in shared memory
             if (abort_sm[buf]) return true;

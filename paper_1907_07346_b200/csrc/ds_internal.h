@@ -13,7 +13,10 @@ namespace ds {
 enum : int { MODE_FUSED = 0, MODE_COMPRESS = 1, MODE_REDUCE = 2 };
 
 // Code formats the kernels are instantiated for.
-enum : int { CODE_SIGN = 0, CODE_U1 = 1, CODE_U2 = 2, CODE_U4 = 3, CODE_U8 = 4, CODE_ID32 = 5 };
+// CODE_N2 / CODE_N4: round-to-nearest b-bit codes whose decoder rescales to the
+// Euclidean norm of the original (the paper's own "bit compression").
+enum : int { CODE_SIGN = 0, CODE_U1 = 1, CODE_U2 = 2, CODE_U4 = 3, CODE_U8 = 4, CODE_ID32 = 5,
+             CODE_N2 = 6, CODE_N4 = 7 };
 
 struct StepParams {
     float* x;
@@ -32,8 +35,10 @@ struct StepParams {
     const float* lut;         // reconstruction levels, 2^bits entries
     uint32_t* codes;
     int64_t code_pitch;       // words
-    float* scales;
+    float* scales;            // the scalar a node sends with each chunk
     int64_t scales_pitch;
+    float* dscales;           // the factor the receiver multiplies the levels by (= scales unless the
+                              // decoder rescales to a norm), same pitch
     double* partials;         // [n][tiles], per-node-scale reduction
     int* error_flag;          // set to 1 by a kernel whose bounded wait ran out
     float sigma;
@@ -70,8 +75,8 @@ cudaError_t launch_noise_kernel(float* out, int32_t n, int64_t N, int64_t ld, in
 inline int code_bits_of(int code) {
     switch (code) {
         case CODE_SIGN: case CODE_U1: return 1;
-        case CODE_U2: return 2;
-        case CODE_U4: return 4;
+        case CODE_U2: case CODE_N2: return 2;
+        case CODE_U4: case CODE_N4: return 4;
         case CODE_U8: return 8;
         default: return 32;
     }

@@ -12,6 +12,8 @@ cudaError_t launch_column_compress(const LaunchShape& sh, const StepParams& p, c
         case CODE_U4: return launch_code<CODE_U4, MODE_COMPRESS>(sh, p, stream);
         case CODE_U8: return launch_code<CODE_U8, MODE_COMPRESS>(sh, p, stream);
         case CODE_ID32: return launch_code<CODE_ID32, MODE_COMPRESS>(sh, p, stream);
+        case CODE_N2: return launch_code<CODE_N2, MODE_COMPRESS>(sh, p, stream);
+        case CODE_N4: return launch_code<CODE_N4, MODE_COMPRESS>(sh, p, stream);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -10,6 +10,8 @@ cudaError_t launch_column_fused(const LaunchShape& sh, const StepParams& p, cuda
         case CODE_U2: return launch_code<CODE_U2, MODE_FUSED>(sh, p, stream);
         case CODE_U4: return launch_code<CODE_U4, MODE_FUSED>(sh, p, stream);
         case CODE_U8: return launch_code<CODE_U8, MODE_FUSED>(sh, p, stream);
+        case CODE_N2: return launch_code<CODE_N2, MODE_FUSED>(sh, p, stream);
+        case CODE_N4: return launch_code<CODE_N4, MODE_FUSED>(sh, p, stream);
         default: return cudaErrorInvalidValue;
     }
 }

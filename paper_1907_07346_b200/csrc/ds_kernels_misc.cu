@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) ds_mix_kernel(const __grid_constant__ Ste
                 for (int t = 0; t < 4; ++t)
                     if (t < nv) acc[t] = __fmaf_rn(w, cf[t], acc[t]);
             } else {
-                const float sj = p.scales[(size_t)j * (size_t)p.scales_pitch + (size_t)tile_idx];
+                const float sj = p.dscales[(size_t)j * (size_t)p.scales_pitch + (size_t)tile_idx];
                 const uint32_t word = cj[f / T::kLanesPerWord];
                 const uint32_t piece = (word >> ((4 * T::kBits * (int)(f % T::kLanesPerWord)) & 31)) & T::kPieceMask;
 #pragma unroll
@@ -79,6 +79,8 @@ cudaError_t launch_mix_kernel(const StepParams& p, int code, cudaStream_t stream
         case CODE_U4: ds_mix_kernel<CODE_U4><<<grid, threads, 0, stream>>>(p); break;
         case CODE_U8: ds_mix_kernel<CODE_U8><<<grid, threads, 0, stream>>>(p); break;
         case CODE_ID32: ds_mix_kernel<CODE_ID32><<<grid, threads, 0, stream>>>(p); break;
+        case CODE_N2: ds_mix_kernel<CODE_N2><<<grid, threads, 0, stream>>>(p); break;
+        case CODE_N4: ds_mix_kernel<CODE_N4><<<grid, threads, 0, stream>>>(p); break;
         default: return cudaErrorInvalidValue;
     }
     return cudaGetLastError();

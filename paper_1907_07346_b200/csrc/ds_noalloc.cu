@@ -94,6 +94,7 @@ extern "C" ds_status ds_node_scales_noalloc(float* scales_out, const float* x, c
     p.lut = reinterpret_cast<const float*>(scratch);          // the zero table
     p.partials = scratch + kTableSlots;
     p.scales = scales_out;
+    p.dscales = scales_out;
     p.scales_pitch = 1;
     p.sigma = gp->sigma;
     p.neg_gamma = -gamma;

@@ -21,6 +21,7 @@ import numpy as np
 COMP_IDENTITY = 0
 COMP_SIGN1_L1 = 1
 COMP_UNIFORM_STOCH_MAXABS = 2
+COMP_UNIFORM_NEAREST_L2 = 3
 
 NOISE_NONE = 0
 NOISE_GAUSS = 1
@@ -136,7 +137,8 @@ class Workload:
 
     def describe(self) -> str:
         comp = {COMP_IDENTITY: "identity", COMP_SIGN1_L1: "1-bit sign l1-scale",
-                COMP_UNIFORM_STOCH_MAXABS: f"{self.bits}-bit uniform stochastic max-abs"}[self.comp_kind]
+                COMP_UNIFORM_STOCH_MAXABS: f"{self.bits}-bit uniform stochastic max-abs",
+                COMP_UNIFORM_NEAREST_L2: f"{self.bits}-bit nearest-level norm-matched"}[self.comp_kind]
         chunk = f"chunk {self.chunk}" if self.chunk else "per-node scale"
         noise = {NOISE_NONE: "none", NOISE_GAUSS: "gauss", NOISE_STUDENT_T3: "student-t3"}[self.noise_kind]
         return (f"{self.name}: n={self.n} {self.graph} N={self.N} {comp} {chunk} "
@@ -154,6 +156,9 @@ WORKLOADS = {
                      NOISE_GAUSS, 0.1, 0.01, 0.5, 50, "uniform", _BASE_SEED + 3),
     "cfg4": Workload("cfg4", 32, "torus4x8", 25_557_032, COMP_UNIFORM_STOCH_MAXABS, 2, 256,
                      NOISE_STUDENT_T3, 0.1, 0.005, 0.4, 50, "uniform", _BASE_SEED + 4),
+    # cfg3's shape with the paper's own codec (Section 5: 4 bits + Euclidean norm, nearest level)
+    "cfg3_l2": Workload("cfg3_l2", 16, "ring", 25_557_032, COMP_UNIFORM_NEAREST_L2, 4, 512,
+                        NOISE_GAUSS, 0.1, 0.01, 0.5, 50, "uniform", _BASE_SEED + 6),
     "cfg5": Workload("cfg5", 64, "exp", 4_194_304, COMP_SIGN1_L1, 1, 1024, NOISE_GAUSS,
                      0.1, 0.01, 0.5, 200, "uniform", _BASE_SEED + 5),
 }

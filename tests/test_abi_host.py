@@ -90,6 +90,9 @@ def test_init_argument_errors():
     assert _init(g, kind=B.DS_COMP_UNIFORM_STOCH_MAXABS, bits=3) == B.DS_ERR_UNSUPPORTED
     assert _init(g, kind=B.DS_COMP_SIGN1_L1, bits=2) == B.DS_ERR_UNSUPPORTED
     assert _init(g, chunk=32768) == B.DS_ERR_UNSUPPORTED
+    assert _init(g, kind=B.DS_COMP_UNIFORM_NEAREST_L2, bits=4, chunk=1024) == B.DS_ERR_UNSUPPORTED
+    assert _init(g, kind=B.DS_COMP_UNIFORM_NEAREST_L2, bits=8, chunk=512) == B.DS_ERR_UNSUPPORTED
+    assert _init(g, kind=B.DS_COMP_UNIFORM_NEAREST_L2, bits=4, chunk=0) == B.DS_ERR_UNSUPPORTED
     assert _init(g, ws_bytes=1024) == B.DS_ERR_WORKSPACE
     st, ctx = B.ds_init_raw(None, g.col_idx, g.w, 8, 1000, 1024, 1, 1, 64, FAKE_WS, BIG)
     assert st == B.DS_ERR_NULL

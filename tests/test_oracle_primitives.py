@@ -293,3 +293,50 @@ def test_pack_layout_and_volume(b):
     assert I.code_words(1 << 20, b) * 32 == (1 << 20) * b
     assert I.code_words(1 << 20, 4) / (1 << 20) == 1 / 8
     assert I.code_words(1 << 20, 2) / (1 << 20) == 1 / 16
+
+
+# ------------------------------- the paper's own compressor (norm-matched)
+@pytest.mark.parametrize("b", [2, 4])
+def test_nearest_l2_compressor(b):
+    """Section 5, "Compression": b bits per element plus the Euclidean norm; the
+    decoded tensor is rescaled to that norm.  Pins: the decoded chunk has the
+    norm that was sent; codes are the nearest grid level (brute force over all
+    levels); C is proportional to the unit levels; b/32 of the volume."""
+    rng = np.random.default_rng(10 + b)
+    L = (1 << b) - 1
+    levels = np.array([orc.level(b, q) for q in range(L + 1)], dtype=np.float64)
+    for m in (1, 9, 64, 512):
+        v = (rng.standard_normal(m) * 10.0 ** rng.uniform(-2, 2)).astype(np.float32)
+        s, q, Cv = orc.compress_chunk(I.COMP_UNIFORM_NEAREST_L2, b, v)
+        v64 = v.astype(np.float64)
+        assert s == pytest.approx(np.sqrt((v64**2).sum()), rel=2e-7)            # what is sent
+        assert np.sqrt((Cv.astype(np.float64)**2).sum()) == pytest.approx(s, rel=1e-6)   # norm matched
+        g = np.abs(v64).max()
+        nearest = np.abs(v64[:, None] / g - levels[None, :]).argmin(axis=1)
+        dist = np.abs(v64[:, None] / g - levels[None, :])
+        ties = np.sort(dist, axis=1)
+        clear = (ties[:, 1] - ties[:, 0]) > 1e-5 if L > 0 else np.ones(m, bool)
+        assert np.array_equal(q[clear], nearest[clear].astype(np.uint32))
+        unit = levels[q]
+        ratio = s / np.sqrt((unit**2).sum())
+        assert np.allclose(Cv, ratio * unit, rtol=3e-7, atol=0)
+    # deterministic: the rounding stream is not used
+    v = rng.standard_normal(100).astype(np.float32)
+    a1 = orc.compress_chunk(I.COMP_UNIFORM_NEAREST_L2, b, v, np.zeros(100, np.float32))
+    a2 = orc.compress_chunk(I.COMP_UNIFORM_NEAREST_L2, b, v, np.full(100, 0.9, np.float32))
+    assert a1[0] == a2[0] and np.array_equal(a1[1], a2[1]) and np.array_equal(a1[2], a2[2])
+    # degenerate chunk
+    s, q, Cv = orc.compress_chunk(I.COMP_UNIFORM_NEAREST_L2, b, np.zeros(7, np.float32))
+    assert s == 0.0 and np.all(q == 0) and np.all(Cv == 0.0)
+
+
+def test_nearest_l2_hand_case():
+    """v = (3, -4, 0, 1) with 2 bits: g = 4, y = (3/4, -1, 0, 1/4), u = 3/2 y + 3/2 =
+    (21/8, 0, 3/2, 15/8), codes floor(u + 1/2) = (3, 0, 2, 2), unit levels (1, -1, 1/3, 1/3),
+    ||v|| = sqrt(26), ||l|| = sqrt(2 + 2/9) = sqrt(20)/3, C = l * 3 sqrt(26/20)."""
+    v = np.array([3.0, -4.0, 0.0, 1.0], dtype=np.float32)
+    s, q, Cv = orc.compress_chunk(I.COMP_UNIFORM_NEAREST_L2, 2, v)
+    assert list(q) == [3, 0, 2, 2]
+    assert s == pytest.approx(np.sqrt(26.0), rel=1e-7)
+    ratio = 3.0 * np.sqrt(26.0 / 20.0)
+    assert np.allclose(Cv, ratio * np.array([1.0, -1.0, 1 / 3, 1 / 3]), rtol=3e-7)

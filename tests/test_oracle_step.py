@@ -15,7 +15,7 @@ GRAPHS = {"ring4": I.ring(4), "ring8": I.ring(8), "torus3x4": I.torus(3, 4),
           "exp16": I.exponential(16)}
 COMPS = [(I.COMP_SIGN1_L1, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 2),
          (I.COMP_UNIFORM_STOCH_MAXABS, 4), (I.COMP_UNIFORM_STOCH_MAXABS, 8),
-         (I.COMP_IDENTITY, 32)]
+         (I.COMP_IDENTITY, 32), (I.COMP_UNIFORM_NEAREST_L2, 2), (I.COMP_UNIFORM_NEAREST_L2, 4)]
 
 
 def make_problem(graph, N, seed, pad=0):
