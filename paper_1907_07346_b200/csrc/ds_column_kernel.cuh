@@ -116,8 +116,10 @@ __device__ __forceinline__ void norm_compress(const float* v, int valid_len, flo
         q[t] = code;
         cv[t] = lut[code];
         if (ok) {
-            sv2 += (double)v[t] * (double)v[t];
-            sl2 += (double)cv[t] * (double)cv[t];
+            // products of two binary32 numbers are exact in binary64, so the fused
+            // form rounds exactly like "sum += product"
+            sv2 = __fma_rn((double)v[t], (double)v[t], sv2);
+            sl2 = __fma_rn((double)cv[t], (double)cv[t], sl2);
         }
     }
 #pragma unroll
