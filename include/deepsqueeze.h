@@ -225,6 +225,16 @@ ds_status ds_get_info(const ds_ctx *ctx, ds_info *info);
  * the step early instead of hanging the device. */
 ds_status ds_sync(ds_ctx *ctx, void *cuda_stream);
 
+/* Arithmetic self-test on the device the library runs on.  The noise kernels
+ * replace two general routines by shortcuts that are exact only on the
+ * arguments that can occur (a branch-free logarithm of j 2^-24 and a
+ * one-correction square root of -2 ln u that starts from the hardware's
+ * reciprocal-square-root estimate).  This runs both against the general forms
+ * on ALL 2^24 possible arguments and ADDS the number of differing results to
+ * counts[0] (logarithms) and counts[1] (square roots); counts is device memory,
+ * two 64-bit integers, zeroed by the caller.  Both must stay 0. */
+ds_status ds_selftest_math(uint64_t *counts, void *cuda_stream);
+
 /* Failure-reporting self-test: enqueues a one-warp kernel that waits, with a
  * small fixed budget, on a completion that never comes, gives up and raises the
  * context's error flag exactly as the fused kernel does when a staged copy does

@@ -24,7 +24,7 @@ DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 
 EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_g", "ds_step_host", "ds_codes", "ds_set_path",
-           "ds_tune", "ds_get_info", "ds_sync", "ds_selftest_timeout", "ds_noise", "ds_node_scales_noalloc",
+           "ds_tune", "ds_get_info", "ds_sync", "ds_selftest_timeout", "ds_selftest_math", "ds_noise", "ds_node_scales_noalloc",
            "ds_destroy", "ds_strerror"]
 
 
@@ -89,6 +89,8 @@ def lib():
         L.ds_sync.restype = C.c_int
         L.ds_selftest_timeout.argtypes = [C.c_void_p, C.c_void_p]
         L.ds_selftest_timeout.restype = C.c_int
+        L.ds_selftest_math.argtypes = [C.c_void_p, C.c_void_p]
+        L.ds_selftest_math.restype = C.c_int
         L.ds_noise.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
                                C.c_uint64, C.c_uint64, C.c_void_p]
         L.ds_noise.restype = C.c_int
@@ -271,3 +273,13 @@ def ds_node_scales_noalloc(scales_out, x, delta, a, c, sigma: float, noise: int,
     return int(lib().ds_node_scales_noalloc(scales_out.data_ptr(), x.data_ptr(), delta.data_ptr(),
                                             C.byref(gp), gamma, n, N, ld, comp_kind, seed, step,
                                             C.c_void_p(s.cuda_stream)))
+
+
+def ds_selftest_math(stream=None):
+    """Run the arithmetic self-test; returns (differing logarithms, differing square roots)."""
+    import torch
+    counts = torch.zeros(2, dtype=torch.int64, device="cuda")
+    s = torch.cuda.current_stream() if stream is None else stream
+    _check(lib().ds_selftest_math(counts.data_ptr(), C.c_void_p(s.cuda_stream)), "ds_selftest_math")
+    torch.cuda.synchronize()
+    return tuple(int(v) for v in counts.cpu())

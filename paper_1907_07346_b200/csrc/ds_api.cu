@@ -501,6 +501,15 @@ ds_status ds_sync(ds_ctx* ctx, void* cuda_stream) {
     return DS_OK;
 }
 
+ds_status ds_selftest_math(uint64_t* counts, void* cuda_stream) {
+    if (!counts) return DS_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(counts) % 8) != 0) return DS_ERR_ALIGN;
+    const cudaError_t e = launch_math_selftest(reinterpret_cast<unsigned long long*>(counts),
+                                               static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+    return DS_OK;
+}
+
 ds_status ds_selftest_timeout(ds_ctx* ctx, void* cuda_stream) {
     if (!ctx) return DS_ERR_NULL;
     const cudaError_t e = launch_wait_selftest(reinterpret_cast<int*>(ctx->base + ctx->ws.error_flag),

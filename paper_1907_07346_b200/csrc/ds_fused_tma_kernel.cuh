@@ -155,6 +155,23 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
 
     int64_t col = blockIdx.x;
     bool pending = (col < p.tiles) ? issue(col) : false;
+    // The gradient noise of a tile depends on nothing that is loaded, so it is
+    // drawn one tile AHEAD (after the mixing of the previous tile): phase A then
+    // only moves the slot into registers and takes the local step, and the refill
+    // of the slot for the next tile is in flight for almost the whole tile time.
+    constexpr bool kNoiseAhead = (NOISE == NOISE_GAUSS || NOISE == NOISE_T3);
+    float zn[kNoiseAhead ? E : 1];
+    auto draw_noise = [&](int64_t c) {
+        if constexpr (kNoiseAhead) {
+#pragma unroll
+            for (int r = 0; r < V; ++r) {
+                const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node,
+                                                (uint32_t)(c * p.tile + seg0 + 4 * (32 * r + lane)));
+                zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
+            }
+        }
+    };
+    if (col < p.tiles) draw_noise(col);
     uint32_t parity = 0;
     int buf = 0;
     constexpr float kL = (float)((1u << (T::kBits & 15)) - 1u);
@@ -199,7 +216,9 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                         local_step4_given(x4, d4, a4, p.neg_gamma, &h[4 * r], &v[4 * r]);
                     } else {
                         const float4 c4 = *reinterpret_cast<const float4*>(slot + 3 * SEG + e0);
-                        const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                        float4 z4;
+                        if constexpr (kNoiseAhead) z4 = make_float4(zn[4 * r + 0], zn[4 * r + 1], zn[4 * r + 2], zn[4 * r + 3]);
+                        else z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
                         local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
                     }
     #pragma unroll
@@ -360,6 +379,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     st_partial(p.x + row + e0, make_float4(xa.x, xa.y, xb.x, xb.y), nv);
                 }
             }
+            if (col + gridDim.x < p.tiles) draw_noise(col + gridDim.x);
             return false;
         };
         const bool aborted = full ? tile_body(std::true_type{}) : tile_body(std::false_type{});

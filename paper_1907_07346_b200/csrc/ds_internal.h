@@ -68,6 +68,7 @@ cudaError_t launch_column_compress(const LaunchShape& shape, const StepParams& p
 cudaError_t launch_column_reduce(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_finalize_scales(const StepParams& p, int code, cudaStream_t stream);
 cudaError_t launch_mix_kernel(const StepParams& p, int code, cudaStream_t stream);
+cudaError_t launch_math_selftest(unsigned long long* counts, cudaStream_t stream);
 cudaError_t launch_wait_selftest(int* error_flag, cudaStream_t stream);
 cudaError_t launch_noise_kernel(float* out, int32_t n, int64_t N, int64_t ld, int which, int noise,
                                 RngStep rs, cudaStream_t stream);

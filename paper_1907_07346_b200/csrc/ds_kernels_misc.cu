@@ -167,6 +167,31 @@ __global__ void __launch_bounds__(32) ds_wait_selftest_kernel(int* error_flag) {
     if (!done && threadIdx.x == 0) *error_flag = 1;
 }
 
+// ---------------------------------------------------------------------------
+// Self-test of the arithmetic shortcuts on every possible argument: the packed
+// branch-free logarithm against the scalar compare-and-halve form, and the
+// one-correction square root against sqrt.rn.f32, for all j = 1 .. 2^24.
+// counts[0] += mismatching logarithms, counts[1] += mismatching roots.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) ds_math_selftest_kernel(unsigned long long* counts) {
+    unsigned bad_log = 0, bad_sqrt = 0;
+    for (uint32_t j = 1u + blockIdx.x * blockDim.x + threadIdx.x; j <= (1u << 24); j += gridDim.x * blockDim.x) {
+        const uint32_t j2 = (j == (1u << 24)) ? 1u : j + 1u;
+        const float2 lg = log_u24_x2(j, j2);
+        if (__float_as_uint(lg.x) != __float_as_uint(log_u24(j))) ++bad_log;
+        if (__float_as_uint(lg.y) != __float_as_uint(log_u24(j2))) ++bad_log;
+        const float t = __fmul_rn(-2.0f, lg.x);
+        if (__float_as_uint(sqrt_of_minus2log(t)) != __float_as_uint(__fsqrt_rn(t))) ++bad_sqrt;
+    }
+    if (bad_log) atomicAdd(&counts[0], (unsigned long long)bad_log);
+    if (bad_sqrt) atomicAdd(&counts[1], (unsigned long long)bad_sqrt);
+}
+
+cudaError_t launch_math_selftest(unsigned long long* counts, cudaStream_t stream) {
+    ds_math_selftest_kernel<<<148 * 8, 256, 0, stream>>>(counts);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_wait_selftest(int* error_flag, cudaStream_t stream) {
     ds_wait_selftest_kernel<<<1, 32, 0, stream>>>(error_flag);
     return cudaGetLastError();

@@ -167,4 +167,5 @@ def test_null_handles():
     assert L.ds_noise(None, 1, 1, 1, 0, 0, 0, 0, None) == B.DS_ERR_NULL
     assert L.ds_sync(None, None) == B.DS_ERR_NULL
     assert L.ds_selftest_timeout(None, None) == B.DS_ERR_NULL
+    assert L.ds_selftest_math(None, None) == B.DS_ERR_NULL
     L.ds_destroy(None)

@@ -116,6 +116,13 @@ def test_rounding_stream_bit_exact(env):
         assert np.array_equal(got[i, :N], orc.rnd24_row(42, i, 9, 0, N))
 
 
+def test_arithmetic_shortcuts_exact_on_all_arguments(env):
+    """The branch-free logarithm and the one-correction square root used by the
+    noise kernels agree bit for bit with the general forms on all 2^24 arguments."""
+    torch, orc, B = env
+    assert B.ds_selftest_math() == (0, 0)
+
+
 # ---------------------------------------------------------- single steps
 COMPS = [(I.COMP_SIGN1_L1, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 2),
          (I.COMP_UNIFORM_STOCH_MAXABS, 4), (I.COMP_UNIFORM_STOCH_MAXABS, 8),
