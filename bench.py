@@ -313,6 +313,8 @@ def main():
                 "algorithmic_bytes_per_update": b_alg,
                 "algorithmic_bytes_per_launch": b_alg * updates_per_step,
                 "kernel_ms_mean": kernel_ms, "kernel_ms_min": min(per_step),
+                "kernel_ms_median": statistics.median(per_step),
+                "kernel_ms_first_last_10": [statistics.mean(per_step[:10]), statistics.mean(per_step[-10:])],
                 "frac_of_nominal_8TBs": achieved / 8000.0}
 
     # End to end through the host-buffer entry point: pinned host arrays in,

@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     volatile int* abort_sm = reinterpret_cast<volatile int*>(smem + L.abort_off);
     const float* slot = reinterpret_cast<const float*>(smem + L.slots_off + (size_t)warp * 4u * L.seg_bytes);
     const uint32_t slot_addr = smem_u32(slot);
+    const float* const slot_lane = slot + 4 * lane;     // this lane's first float4 of each staged array
     const uint32_t bar = smem_u32(smem + L.mbar_off + warp * 8);
 
     if constexpr (T::kLut)
@@ -209,13 +210,13 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 const int e0 = 4 * (32 * r + lane);              // offset inside the segment
                 const int nv = FULL ? 4 : min(max(live_len - e0, 0), 4);
                 if (nv > 0) {
-                    const float4 x4 = *reinterpret_cast<const float4*>(slot + 0 * SEG + e0);
-                    const float4 d4 = *reinterpret_cast<const float4*>(slot + 1 * SEG + e0);
-                    const float4 a4 = *reinterpret_cast<const float4*>(slot + 2 * SEG + e0);
+                    const float4 x4 = *reinterpret_cast<const float4*>(slot_lane + 0 * SEG + 128 * r);
+                    const float4 d4 = *reinterpret_cast<const float4*>(slot_lane + 1 * SEG + 128 * r);
+                    const float4 a4 = *reinterpret_cast<const float4*>(slot_lane + 2 * SEG + 128 * r);
                     if constexpr (NOISE == GRAD_GIVEN) {
                         local_step4_given(x4, d4, a4, p.neg_gamma, &h[4 * r], &v[4 * r]);
                     } else {
-                        const float4 c4 = *reinterpret_cast<const float4*>(slot + 3 * SEG + e0);
+                        const float4 c4 = *reinterpret_cast<const float4*>(slot_lane + 3 * SEG + 128 * r);
                         float4 z4;
                         if constexpr (kNoiseAhead) z4 = make_float4(zn[4 * r + 0], zn[4 * r + 1], zn[4 * r + 2], zn[4 * r + 3]);
                         else z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
@@ -270,6 +271,11 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             const float inv_s = fast ? __fdiv_rn(1.0f, s) : 0.0f;
             const size_t code_row = (size_t)node * (size_t)p.code_pitch + (size_t)(((k0 + seg0) * T::kBits) >> 5);
             float* cval_mine = cval + (size_t)node * p.tile + seg0;
+            // per-lane bases: element 4*(32*r + lane) of the segment is base + 128*r
+            float* const cval_lane = cval_mine + 4 * lane;
+            float* const delta_lane = p.delta + row + 4 * lane;
+            float* const x_lane = p.x + row + 4 * lane;
+            uint32_t* const codes_lane = p.codes + code_row + lane / T::kLanesPerWord;
             // norm-matched codes: the whole chunk is coded first (two more warp
             // reductions), s becomes the norm that is sent, dscale the decode factor
             uint32_t qn[T::kNorm ? E : 1];
@@ -329,14 +335,14 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                         const float2 db = __fadd2_rn(make_float2(v[4 * r + 2], v[4 * r + 3]), make_float2(-cv[2], -cv[3]));
                         dn[0] = da.x; dn[1] = da.y; dn[2] = db.x; dn[3] = db.y;
                     }
-                    st_partial(p.delta + row + e0, make_float4(dn[0], dn[1], dn[2], dn[3]), nv);
-                    *reinterpret_cast<float4*>(cval_mine + e0) = make_float4(cv[0], cv[1], cv[2], cv[3]);
+                    st_partial(delta_lane + 128 * r, make_float4(dn[0], dn[1], dn[2], dn[3]), nv);
+                    *reinterpret_cast<float4*>(cval_lane + 128 * r) = make_float4(cv[0], cv[1], cv[2], cv[3]);
                 }
                 uint32_t word = piece << ((4 * T::kBits * (lane % T::kLanesPerWord)) & 31);
     #pragma unroll
                 for (int o = 1; o < T::kLanesPerWord; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
                 if ((lane % T::kLanesPerWord) == 0 && (FULL || e0 < live_len))
-                    p.codes[code_row + f / T::kLanesPerWord] = word;
+                    codes_lane[(32 / T::kLanesPerWord) * r] = word;
             }
             if (!p.prescaled && alive && wg == 0 && lane == 0)
             {
@@ -359,7 +365,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 for (int r = 0; r < V; ++r) {
                     const int e0 = 4 * (32 * r + lane);
                     if (!FULL && e0 >= live_len) continue;
-                    const float4 c4 = *reinterpret_cast<const float4*>(cn + e0);
+                    const float4 c4 = *reinterpret_cast<const float4*>(cn + 4 * lane + 128 * r);
                     {
                         const float2 w2 = splat(w);
                         const float2 aa = __ffma2_rn(w2, make_float2(c4.x, c4.y), make_float2(acc[4 * r + 0], acc[4 * r + 1]));
@@ -376,7 +382,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     const float2 et = splat(p.eta);
                     const float2 xa = __ffma2_rn(et, make_float2(acc[4 * r + 0], acc[4 * r + 1]), make_float2(h[4 * r + 0], h[4 * r + 1]));
                     const float2 xb = __ffma2_rn(et, make_float2(acc[4 * r + 2], acc[4 * r + 3]), make_float2(h[4 * r + 2], h[4 * r + 3]));
-                    st_partial(p.x + row + e0, make_float4(xa.x, xa.y, xb.x, xb.y), nv);
+                    st_partial(x_lane + 128 * r, make_float4(xa.x, xa.y, xb.x, xb.y), nv);
                 }
             }
             if (col + gridDim.x < p.tiles) draw_noise(col + gridDim.x);
