@@ -162,7 +162,18 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     // of the slot for the next tile is in flight for almost the whole tile time.
     constexpr bool kNoiseAhead = (NOISE == NOISE_GAUSS || NOISE == NOISE_T3);
     float zn[kNoiseAhead ? E : 1];
+    // the rounding uniforms of the stochastic quantiser are drawn with it
+    constexpr bool kRndAhead = T::kLut && !T::kNorm;
+    float mn[kRndAhead ? E : 1];
     auto draw_noise = [&](int64_t c) {
+        if constexpr (kRndAhead) {
+#pragma unroll
+            for (int r = 0; r < V; ++r) {
+                const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node,
+                                                   (uint32_t)(c * p.tile + seg0 + 4 * (32 * r + lane)));
+                mn[4 * r + 0] = rr.x; mn[4 * r + 1] = rr.y; mn[4 * r + 2] = rr.z; mn[4 * r + 3] = rr.w;
+            }
+        }
         if constexpr (kNoiseAhead) {
 #pragma unroll
             for (int r = 0; r < V; ++r) {
@@ -172,7 +183,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             }
         }
     };
-    if (col < p.tiles) draw_noise(col);
+    if (col < p.tiles) draw_noise(col);      // (also when only the rounding stream is needed)
     uint32_t parity = 0;
     int buf = 0;
     constexpr float kL = (float)((1u << (T::kBits & 15)) - 1u);
@@ -310,7 +321,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                             if (FULL || j < nv) piece |= bit << j;
                         }
                     } else if (fast) {
-                        const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
+                        const float4 rr = make_float4(mn[4 * r + 0], mn[4 * r + 1], mn[4 * r + 2], mn[4 * r + 3]);
                         uint32_t q[4];
                         quantise_recip2(v[4 * r + 0], v[4 * r + 1], s, inv_s, rr.x, rr.y, kHalfL, (int)kL, q[0], q[1]);
                         quantise_recip2(v[4 * r + 2], v[4 * r + 3], s, inv_s, rr.z, rr.w, kHalfL, (int)kL, q[2], q[3]);
@@ -321,8 +332,8 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                         for (int j = 0; j < 4; ++j)
                             if (FULL || j < nv) piece |= q[j] << (T::kBits * j);
                     } else {
-                        const float4 rr = rnd24x4(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
-                        const float rv[4] = {rr.x, rr.y, rr.z, rr.w};
+                        const float rv[4] = {__fmul_rn(mn[4 * r + 0], 0x1p-24f), __fmul_rn(mn[4 * r + 1], 0x1p-24f),
+                                             __fmul_rn(mn[4 * r + 2], 0x1p-24f), __fmul_rn(mn[4 * r + 3], 0x1p-24f)};
     #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const uint32_t q = degenerate ? 0u : quantise(v[4 * r + j], s, rv[j], kHalfL, (int)kL);
