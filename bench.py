@@ -238,7 +238,7 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
-    if world > 1:
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:      # launched by torch.distributed.run
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
