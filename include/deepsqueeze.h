@@ -64,8 +64,9 @@ typedef struct {
 
 /* Compressor C_omega (Algorithm 1, compression step; Section 5, "Compression":
  * every element is sent with b bits plus one scalar per tensor).
- *   DS_COMP_IDENTITY             C[v] = v (D-PSGD, Section 3.2); the "codes" are the
- *                                bit patterns of v, 32 bits per element; bits is ignored.
+ *   DS_COMP_IDENTITY             C[v] = v: no compression, i.e. D-PSGD (Section 3.2), the
+ *                                baseline the paper compares with; the "codes" are the bit
+ *                                patterns of v, 32 bits per element; bits is ignored.
  *   DS_COMP_SIGN1_L1             one bit per element: bit = (v >= 0); C = +s / -s with
  *                                s = (sum |v|)/m over the chunk (binary64 sum); bits must be 1.
  *   DS_COMP_UNIFORM_STOCH_MAXABS b in {1,2,4,8} bits: 2^b levels evenly spaced on

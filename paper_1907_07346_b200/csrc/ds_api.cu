@@ -139,13 +139,13 @@ Plan plan_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int force_e 
     pick_lane_shape(sh.tile, force_e, &E, &G);
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
-    if (sh.code == CODE_ID32 || (int64_t)n * G > 32 || num_sms < 1) return pl;
+    if ((int64_t)n * G > 32 || num_sms < 1) return pl;
     if ((sh.code == CODE_N2 || sh.code == CODE_N4) && G != 1) return pl;
     // every warp of a group owns a whole E*32-element segment
     if ((int64_t)G * E * 32 < sh.tile) return pl;
     pl.nodes_per_block = n;
     pl.block = dim3((unsigned)(n * G * 32));
-    const bool lut = (sh.code != CODE_SIGN);
+    const bool lut = (sh.code != CODE_SIGN && sh.code != CODE_ID32);
     pl.smem = tma_smem_layout(lut, E, n * G, G, sh.tile, n, nnz).total;
     if (pl.smem > (size_t)kMaxSmem) return pl;
     pl.grid = dim3((unsigned)std::min<int64_t>(sh.tiles, num_sms));

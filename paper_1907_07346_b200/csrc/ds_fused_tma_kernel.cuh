@@ -99,7 +99,6 @@ __device__ __forceinline__ void fence_proxy_async() {
 template <int CODE, int NOISE, int E, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_constant__ StepParams p) {
     using T = CodeTraits<CODE>;
-    static_assert(!T::kIdentity, "the identity compressor runs on the two-kernel path");
     constexpr int V = E / 4;
     constexpr int SEG = E * 32;                       // elements per warp segment
     extern __shared__ __align__(128) unsigned char smem[];
@@ -237,7 +236,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     for (int j = 0; j < 4; ++j) {
                         if (!FULL && j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
                         if constexpr (T::kSign) sum += (double)fabsf(v[4 * r + j]);
-                        else mx = fmaxf(mx, fabsf(v[4 * r + j]));
+                        else if constexpr (!T::kIdentity) mx = fmaxf(mx, fabsf(v[4 * r + j]));
                     }
                 } else {
     #pragma unroll
@@ -253,7 +252,9 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
 
             // ---- scale of the (node, tile) -----------------------------------
             float s;
-            if (p.prescaled) {
+            if constexpr (T::kIdentity) {
+                s = 1.0f;                       // C[v] = v: nothing to scale
+            } else if (p.prescaled) {
                 s = p.scales[(size_t)node * (size_t)p.scales_pitch];
             } else {
                 double part;
@@ -307,7 +308,13 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 uint32_t piece = 0u;
                 if (nv > 0) {
                     float dn[4], cv[4];
-                    if constexpr (T::kNorm) {
+                    if constexpr (T::kIdentity) {
+                        // D-PSGD: what is sent is v itself (32 bits per element)
+    #pragma unroll
+                        for (int j = 0; j < 4; ++j) cv[j] = v[4 * r + j];
+                        st_partial(reinterpret_cast<float*>(p.codes + code_row) + e0,
+                                   make_float4(cv[0], cv[1], cv[2], cv[3]), nv);
+                    } else if constexpr (T::kNorm) {
     #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             cv[j] = cvn[4 * r + j];
@@ -352,10 +359,12 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 uint32_t word = piece << ((4 * T::kBits * (lane % T::kLanesPerWord)) & 31);
     #pragma unroll
                 for (int o = 1; o < T::kLanesPerWord; o <<= 1) word |= __shfl_xor_sync(0xffffffffu, word, o);
-                if ((lane % T::kLanesPerWord) == 0 && (FULL || e0 < live_len))
-                    codes_lane[(32 / T::kLanesPerWord) * r] = word;
+                if constexpr (!T::kIdentity) {
+                    if ((lane % T::kLanesPerWord) == 0 && (FULL || e0 < live_len))
+                        codes_lane[(32 / T::kLanesPerWord) * r] = word;
+                }
             }
-            if (!p.prescaled && alive && wg == 0 && lane == 0)
+            if (!T::kIdentity && !p.prescaled && alive && wg == 0 && lane == 0)
             {
                 p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
                 if constexpr (T::kNorm) p.dscales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = dscale;

@@ -10,6 +10,7 @@ cudaError_t launch_fused_tma(const LaunchShape& sh, const StepParams& p, cudaStr
         case CODE_U2: return launch_tma_code<CODE_U2>(sh, p, stream);
         case CODE_U4: return launch_tma_code<CODE_U4>(sh, p, stream);
         case CODE_U8: return launch_tma_code<CODE_U8>(sh, p, stream);
+        case CODE_ID32: return launch_tma_code<CODE_ID32>(sh, p, stream);
         case CODE_N2: return launch_tma_code<CODE_N2>(sh, p, stream);
         case CODE_N4: return launch_tma_code<CODE_N4>(sh, p, stream);
         default: return cudaErrorInvalidValue;

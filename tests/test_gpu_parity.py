@@ -167,6 +167,9 @@ def test_identity_compressor(env):
     torch, orc, B = env
     run_case(env, I.ring(8), 1000, I.COMP_IDENTITY, 32, 0, I.NOISE_GAUSS, B.DS_PATH_SPLIT)
     run_case(env, I.exponential(16), 999, I.COMP_IDENTITY, 32, 64, I.NOISE_NONE, B.DS_PATH_SPLIT)
+    # D-PSGD on the persistent fused kernel
+    run_case(env, I.ring(8), 512 * 3 + 11, I.COMP_IDENTITY, 32, 0, I.NOISE_GAUSS, B.DS_PATH_FUSED, steps=3)
+    run_case(env, I.ring(16), 512 * 4 + 40, I.COMP_IDENTITY, 32, 512, I.NOISE_STUDENT_T3, B.DS_PATH_FUSED)
 
 
 @pytest.mark.parametrize("path", PATHS)
@@ -359,3 +362,22 @@ def test_norm_matched_compressor_free_running(env, path, bits):
              steps=20, zero_start=True, tol=TOL_RUN, gamma=0.01)
     run_case(env, I.torus(4, 8), 256 * 5 + 7, I.COMP_UNIFORM_NEAREST_L2, bits, 256, I.NOISE_STUDENT_T3, path,
              steps=3)
+
+
+def test_compressed_runs_track_the_uncompressed_baseline(env):
+    """The paper's qualitative result on its topology (8 workers on a ring): with
+    error compensation, 4-bit compression converges like uncompressed D-PSGD and
+    2-bit somewhat slower but still converges (Section 5.2)."""
+    import argparse
+    from paper_1907_07346_b200 import demo_convergence
+    args = argparse.Namespace(nodes=8, params=8192, steps=300, gamma=0.05, eta=0.4, sigma=0.1)
+    res = {name: (dist, cons) for name, bits, dist, cons, dn in demo_convergence.run(args)}
+    base = res["none (D-PSGD)"][0]
+    assert base < 0.2
+    assert res["4-bit stochastic"][0] < base + 0.02
+    assert res["4-bit nearest + norm"][0] < base + 0.03
+    assert res["2-bit stochastic"][0] < base + 0.1
+    assert res["2-bit nearest + norm"][0] < base + 0.15
+    assert res["1-bit sign"][0] < 0.6
+    for dist, cons in res.values():
+        assert np.isfinite(dist) and np.isfinite(cons)
