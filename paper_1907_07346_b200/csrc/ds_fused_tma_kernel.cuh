@@ -165,20 +165,38 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     constexpr bool kRndAhead = T::kLut && !T::kNorm;
     float mn[kRndAhead ? E : 1];
     auto draw_noise = [&](int64_t c) {
-        if constexpr (kRndAhead) {
+        const uint32_t kbase = (uint32_t)(c * p.tile + seg0) + 4u * (uint32_t)lane;   // element of r = 0
+        if constexpr (NOISE == NOISE_GAUSS && kRndAhead) {
+            // the 2V Philox blocks of the tile (noise and rounding) advance together
+            uint32_t stream[2 * V], block[2 * V];
+            uint4 w[2 * V];
 #pragma unroll
             for (int r = 0; r < V; ++r) {
-                const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node,
-                                                   (uint32_t)(c * p.tile + seg0 + 4 * (32 * r + lane)));
-                mn[4 * r + 0] = rr.x; mn[4 * r + 1] = rr.y; mn[4 * r + 2] = rr.z; mn[4 * r + 3] = rr.w;
+                stream[r] = STREAM_NOISE; stream[V + r] = STREAM_ROUND;
+                block[r] = block[V + r] = (kbase + 128u * (uint32_t)r) >> 2;
             }
-        }
-        if constexpr (kNoiseAhead) {
+            rng_blocks<2 * V>(p.rs, (uint32_t)node, stream, block, w);
 #pragma unroll
             for (int r = 0; r < V; ++r) {
-                const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node,
-                                                (uint32_t)(c * p.tile + seg0 + 4 * (32 * r + lane)));
+                const float4 z4 = box_muller_x2(w[r]);
                 zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
+                mn[4 * r + 0] = __uint2float_rn(w[V + r].x >> 8); mn[4 * r + 1] = __uint2float_rn(w[V + r].y >> 8);
+                mn[4 * r + 2] = __uint2float_rn(w[V + r].z >> 8); mn[4 * r + 3] = __uint2float_rn(w[V + r].w >> 8);
+            }
+        } else {
+            if constexpr (kRndAhead) {
+#pragma unroll
+                for (int r = 0; r < V; ++r) {
+                    const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node, kbase + 128u * (uint32_t)r);
+                    mn[4 * r + 0] = rr.x; mn[4 * r + 1] = rr.y; mn[4 * r + 2] = rr.z; mn[4 * r + 3] = rr.w;
+                }
+            }
+            if constexpr (kNoiseAhead) {
+#pragma unroll
+                for (int r = 0; r < V; ++r) {
+                    const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, kbase + 128u * (uint32_t)r);
+                    zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
+                }
             }
         }
     };
