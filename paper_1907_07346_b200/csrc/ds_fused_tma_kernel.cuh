@@ -183,6 +183,20 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 mn[4 * r + 0] = __uint2float_rn(w[V + r].x >> 8); mn[4 * r + 1] = __uint2float_rn(w[V + r].y >> 8);
                 mn[4 * r + 2] = __uint2float_rn(w[V + r].z >> 8); mn[4 * r + 3] = __uint2float_rn(w[V + r].w >> 8);
             }
+        } else if constexpr (NOISE == NOISE_T3 && kRndAhead) {
+            // per four elements: their four noise blocks and the rounding block together
+#pragma unroll
+            for (int r = 0; r < V; ++r) {
+                const uint32_t kr = kbase + 128u * (uint32_t)r;
+                const uint32_t stream[5] = {STREAM_NOISE, STREAM_NOISE, STREAM_NOISE, STREAM_NOISE, STREAM_ROUND};
+                const uint32_t block[5] = {kr, kr + 1u, kr + 2u, kr + 3u, kr >> 2};
+                uint4 w[5];
+                rng_blocks<5>(p.rs, (uint32_t)node, stream, block, w);
+                student_t3_pair(w[0], w[1], zn[4 * r + 0], zn[4 * r + 1]);
+                student_t3_pair(w[2], w[3], zn[4 * r + 2], zn[4 * r + 3]);
+                mn[4 * r + 0] = __uint2float_rn(w[4].x >> 8); mn[4 * r + 1] = __uint2float_rn(w[4].y >> 8);
+                mn[4 * r + 2] = __uint2float_rn(w[4].z >> 8); mn[4 * r + 3] = __uint2float_rn(w[4].w >> 8);
+            }
         } else {
             if constexpr (kRndAhead) {
 #pragma unroll
