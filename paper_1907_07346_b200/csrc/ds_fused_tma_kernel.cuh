@@ -166,22 +166,30 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     float mn[kRndAhead ? E : 1];
     auto draw_noise = [&](int64_t c) {
         const uint32_t kbase = (uint32_t)(c * p.tile + seg0) + 4u * (uint32_t)lane;   // element of r = 0
-        if constexpr (NOISE == NOISE_GAUSS && kRndAhead) {
-            // the 2V Philox blocks of the tile (noise and rounding) advance together
-            uint32_t stream[2 * V], block[2 * V];
-            uint4 w[2 * V];
+        if constexpr (NOISE == NOISE_GAUSS || (NOISE != NOISE_T3 && kRndAhead)) {
+            // all Philox blocks of the tile (V for the noise, V for the rounding stream,
+            // whichever are needed) advance together
+            constexpr int kGauss = (NOISE == NOISE_GAUSS) ? V : 0;
+            constexpr int kRnd = kRndAhead ? V : 0;
+            uint32_t stream[kGauss + kRnd], block[kGauss + kRnd];
+            uint4 w[kGauss + kRnd];
 #pragma unroll
             for (int r = 0; r < V; ++r) {
-                stream[r] = STREAM_NOISE; stream[V + r] = STREAM_ROUND;
-                block[r] = block[V + r] = (kbase + 128u * (uint32_t)r) >> 2;
+                if constexpr (kGauss > 0) { stream[r] = STREAM_NOISE; block[r] = (kbase + 128u * (uint32_t)r) >> 2; }
+                if constexpr (kRnd > 0) { stream[kGauss + r] = STREAM_ROUND; block[kGauss + r] = (kbase + 128u * (uint32_t)r) >> 2; }
             }
-            rng_blocks<2 * V>(p.rs, (uint32_t)node, stream, block, w);
+            rng_blocks<kGauss + kRnd>(p.rs, (uint32_t)node, stream, block, w);
 #pragma unroll
             for (int r = 0; r < V; ++r) {
-                const float4 z4 = box_muller_x2(w[r]);
-                zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
-                mn[4 * r + 0] = __uint2float_rn(w[V + r].x >> 8); mn[4 * r + 1] = __uint2float_rn(w[V + r].y >> 8);
-                mn[4 * r + 2] = __uint2float_rn(w[V + r].z >> 8); mn[4 * r + 3] = __uint2float_rn(w[V + r].w >> 8);
+                if constexpr (kGauss > 0) {
+                    const float4 z4 = box_muller_x2(w[r]);
+                    zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
+                }
+                if constexpr (kRnd > 0) {
+                    const uint4 u = w[kGauss + r];
+                    mn[4 * r + 0] = __uint2float_rn(u.x >> 8); mn[4 * r + 1] = __uint2float_rn(u.y >> 8);
+                    mn[4 * r + 2] = __uint2float_rn(u.z >> 8); mn[4 * r + 3] = __uint2float_rn(u.w >> 8);
+                }
             }
         } else if constexpr (NOISE == NOISE_T3 && kRndAhead) {
             // per four elements: their four noise blocks and the rounding block together
