@@ -381,3 +381,37 @@ def test_compressed_runs_track_the_uncompressed_baseline(env):
     assert res["1-bit sign"][0] < 0.6
     for dist, cons in res.values():
         assert np.isfinite(dist) and np.isfinite(cons)
+
+
+def test_results_do_not_depend_on_tuning_or_stream(env):
+    """Elements per lane (4, 8, 16), the execution path and the stream are
+    scheduling choices: x, delta, codes and scales come out bit-identical."""
+    torch, orc, B = env
+    g = I.ring(16)
+    N, ld = 512 * 7 + 40, 512 * 7 + 40
+    x, d, a, c = make_state(g, N, ld, 12)
+    outs = []
+    side = torch.cuda.Stream()
+    for path, e, stream in [(B.DS_PATH_FUSED, 0, None), (B.DS_PATH_FUSED, 8, None), (B.DS_PATH_FUSED, 4, side),
+                            (B.DS_PATH_FUSED_LDG, 8, None), (B.DS_PATH_SPLIT, 4, side)]:
+        ds = B.DeepSqueeze(g, N, ld, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512)
+        ds.ds_tune(e)
+        ds.ds_set_path(path)
+        dev = [torch.from_numpy(t.copy()).cuda() for t in (x, d, a, c)]
+        torch.cuda.synchronize()
+        for t in range(3):
+            ds.ds_step(dev[0], dev[1], dev[2], dev[3], 0.1, I.NOISE_GAUSS, 0.01, 0.5, 21, t, stream)
+        ds.ds_sync(stream)
+        outs.append((dev[0].cpu().numpy(), dev[1].cpu().numpy(), *ds.codes_to_host()))
+        ds.close()
+    for other in outs[1:]:
+        for u, v in zip(outs[0], other):
+            assert np.array_equal(u, v)
+
+
+@pytest.mark.parametrize("path", [3, 2])
+def test_many_nodes(env, path):
+    """200 nodes on a ring: far more than one block holds (node batches on the
+    wide kernel, many grid rows on the two-kernel path)."""
+    run_case(env, I.ring(200), 512 + 72, I.COMP_UNIFORM_STOCH_MAXABS, 2, 256, I.NOISE_GAUSS, path)
+    run_case(env, I.ring(200), 1024 + 33, I.COMP_SIGN1_L1, 1, 1024, I.NOISE_NONE, path)
