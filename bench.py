@@ -341,7 +341,8 @@ def main():
         e2e = {"value": whole_job_value(world, updates_per_step, args.e2e_steps, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": 4 * arr_bytes, "d2h_bytes_per_step": 2 * arr_bytes,
                "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
-               "entry_point": "ds_step_host (pinned host x, delta, a, c in; x, delta out)"}
+               "entry_point": "ds_step_host (pinned host x, delta, a, c in; x, delta out; slabs of column tiles "
+                              "pipelined: copy in / compute / copy out overlap)"}
         del hx, hd, ha, hc
 
     base = None

@@ -185,12 +185,16 @@ ds_status ds_step(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
 ds_status ds_step_g(ds_ctx *ctx, float *x, float *delta, const float *g, const ds_hparams *hp,
                     uint64_t seed, uint64_t step, void *cuda_stream);
 
-/* Same iteration for HOST buffers: copies x, delta, a, c (host, [n][ld]) into
- * the caller's device staging arrays, runs ds_step, and copies x and delta
- * back, all enqueued on `cuda_stream`; the caller synchronises the stream
- * before reading the results.  Host buffers should be page-locked for the
- * copies to be asynchronous.  dev_* are device [n][ld] arrays owned by the
- * caller. */
+/* Same iteration for HOST buffers: x, delta, a, c (host, [n][ld]) go to the
+ * caller's device staging arrays, the step runs, and x and delta come back,
+ * all ordered after the work already in `cuda_stream`; that stream continues
+ * once the results are back, and the caller synchronises it before reading
+ * them.  Host buffers must be page-locked for the copies to overlap.  Unless
+ * one scale covers a whole node (chunk = 0), the work is cut into slabs of
+ * column tiles and pipelined on three internal streams (created at the first
+ * call): while one slab is computed the next is on its way in and the previous
+ * on its way out.  Padding columns are copied in, never out.  dev_* are device
+ * [n][ld] arrays owned by the caller.  Only the synthetic objective. */
 ds_status ds_step_host(ds_ctx *ctx, float *x_host, float *delta_host,
                        const float *a_host, const float *c_host,
                        float sigma, int32_t noise, const ds_hparams *hp,

@@ -17,6 +17,7 @@ namespace {
 constexpr size_t kAlign = 256;
 constexpr int64_t kPerNodeTile = 512;   // tile width when one scale covers a node
 constexpr int kMaxSmem = 227 * 1024;
+constexpr int kMaxSlabs = 16;            // pipeline depth of the host-buffer entry point
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int64_t round_up64(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
@@ -184,6 +185,9 @@ struct ds_ctx {
     int path_req;
     Plan tma, fused, wide, compress, reduce;
     int num_sms;
+    bool pipe_ready;                                  // streams / events of ds_step_host
+    cudaStream_t pipe_stream[3];
+    cudaEvent_t pipe_event[2 * kMaxSlabs + 2];
 };
 
 extern "C" {
@@ -275,6 +279,7 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     ctx->comp = *comp; ctx->sh = sh; ctx->ws = ws;
     ctx->base = static_cast<unsigned char*>(workspace);
     ctx->path_req = DS_PATH_AUTO;
+    ctx->pipe_ready = false;
     ctx->compress = plan_column(MODE_COMPRESS, sh, n, nnz);
     ctx->reduce = plan_column(MODE_REDUCE, sh, n, nnz);
     if (!ctx->compress.ok) { delete ctx; return DS_ERR_UNSUPPORTED; }
@@ -317,7 +322,14 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     return DS_OK;
 }
 
-void ds_destroy(ds_ctx* ctx) { delete ctx; }
+void ds_destroy(ds_ctx* ctx) {
+    if (!ctx) return;
+    if (ctx->pipe_ready) {
+        for (int i = 0; i < 3; ++i) (void)cudaStreamDestroy(ctx->pipe_stream[i]);
+        for (int i = 0; i < 2 * kMaxSlabs + 2; ++i) (void)cudaEventDestroy(ctx->pipe_event[i]);
+    }
+    delete ctx;
+}
 
 // 2: persistent TMA-staged fused kernel, 1: fused kernel with direct loads,
 // 3: the same in node batches (wide columns), 0: two kernels
@@ -382,8 +394,9 @@ ds_status ds_codes(ds_ctx* ctx, const uint32_t** codes, int64_t* code_pitch_word
 // (a, c given) or GRAD_GIVEN (a is the gradient itself, c unused).
 static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, const float* c,
                           float sigma, int grad_kind, const ds_hparams* hp, uint64_t seed,
-                          uint64_t step, void* cuda_stream) {
+                          uint64_t step, void* cuda_stream, int64_t tile_begin = 0, int64_t tile_end = -1) {
     if (step >= ((uint64_t)1 << 56)) return DS_ERR_ARG;
+    if (tile_end < 0) tile_end = ctx->sh.tiles;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
                            reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(c);
     if ((bits % 16) != 0) return DS_ERR_ALIGN;
@@ -393,6 +406,7 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
     p.x = x; p.delta = delta; p.a = a; p.c = c;
     p.ld = ctx->ld; p.N = ctx->N; p.n = ctx->n; p.nnz = ctx->nnz;
     p.tile = ctx->sh.tile; p.tiles = ctx->sh.tiles;
+    p.tile_begin = tile_begin; p.tile_end = tile_end;
     p.row_ptr = reinterpret_cast<const int32_t*>(ctx->base + ctx->ws.row_ptr);
     p.col_idx = reinterpret_cast<const int32_t*>(ctx->base + ctx->ws.col_idx);
     p.wprime = reinterpret_cast<const float*>(ctx->base + ctx->ws.wprime);
@@ -414,6 +428,8 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
         LaunchShape s;
         s.code = ctx->sh.code; s.noise = grad_kind; s.elems_per_lane = pl.elems_per_lane;
         s.mode = mode; s.grid = pl.grid; s.block = pl.block; s.smem = pl.smem;
+        // a launch over part of the tiles needs no more blocks than tiles
+        s.grid.x = (unsigned)std::max<int64_t>(1, std::min<int64_t>(pl.grid.x, tile_end - tile_begin));
         return s;
     };
     cudaError_t e = cudaSuccess;
@@ -464,6 +480,19 @@ ds_status ds_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, const d
     return run_step(ctx, x, delta, g, nullptr, 0.0f, GRAD_GIVEN, hp, seed, step, cuda_stream);
 }
 
+// Streams and events of the host-buffer entry point, made on first use.
+static bool ensure_pipeline(ds_ctx* ctx) {
+    if (ctx->pipe_ready) return true;
+    bool ok = true;
+    for (int i = 0; i < 3 && ok; ++i)
+        ok = cudaStreamCreateWithFlags(&ctx->pipe_stream[i], cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < 2 * kMaxSlabs + 2 && ok; ++i)
+        ok = cudaEventCreateWithFlags(&ctx->pipe_event[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) { (void)cudaGetLastError(); return false; }
+    ctx->pipe_ready = true;
+    return true;
+}
+
 ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const float* a_host,
                        const float* c_host, float sigma, int32_t noise, const ds_hparams* hp,
                        uint64_t seed, uint64_t step, float* dev_x, float* dev_delta, float* dev_a,
@@ -471,19 +500,65 @@ ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const floa
     if (!ctx || !x_host || !delta_host || !a_host || !c_host || !hp || !dev_x || !dev_delta ||
         !dev_a || !dev_c)
         return DS_ERR_NULL;
+    if (noise < DS_NOISE_NONE || noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const size_t bytes = (size_t)ctx->n * (size_t)ctx->ld * sizeof(float);
-    cudaError_t e = cudaMemcpyAsync(dev_x, x_host, bytes, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(dev_delta, delta_host, bytes, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(dev_a, a_host, bytes, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(dev_c, c_host, bytes, cudaMemcpyHostToDevice, stream);
-    if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
-    ds_grad_params gp;
-    gp.a = dev_a; gp.c = dev_c; gp.sigma = sigma; gp.noise = noise;
-    const ds_status st = ds_step(ctx, dev_x, dev_delta, &gp, hp, seed, step, cuda_stream);
-    if (st != DS_OK) return st;
-    e = cudaMemcpyAsync(x_host, dev_x, bytes, cudaMemcpyDeviceToHost, stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(delta_host, dev_delta, bytes, cudaMemcpyDeviceToHost, stream);
+    const size_t pitch = (size_t)ctx->ld * sizeof(float);
+    const size_t bytes = (size_t)ctx->n * pitch;
+
+    // Column tiles are independent unless one scale covers a whole node, so the
+    // step is cut into slabs of tiles and pipelined: slab s+1 travels to the
+    // device while slab s is computed and slab s-1 travels back (PCIe carries
+    // both directions at once).
+    const int64_t tiles = ctx->sh.tiles;
+    int slabs = 1;
+    if (!ctx->sh.per_node && bytes >= ((size_t)64 << 20)) slabs = (int)std::min<int64_t>(kMaxSlabs, tiles);
+    if (slabs == 1 || !ensure_pipeline(ctx)) {
+        cudaError_t e = cudaMemcpyAsync(dev_x, x_host, bytes, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dev_delta, delta_host, bytes, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dev_a, a_host, bytes, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dev_c, c_host, bytes, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+        const ds_status st = run_step(ctx, dev_x, dev_delta, dev_a, dev_c, sigma, noise, hp, seed, step, cuda_stream);
+        if (st != DS_OK) return st;
+        e = cudaMemcpyAsync(x_host, dev_x, bytes, cudaMemcpyDeviceToHost, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(delta_host, dev_delta, bytes, cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+        return DS_OK;
+    }
+
+    cudaStream_t s_in = ctx->pipe_stream[0], s_run = ctx->pipe_stream[1], s_out = ctx->pipe_stream[2];
+    cudaEvent_t ev_start = ctx->pipe_event[2 * kMaxSlabs], ev_done = ctx->pipe_event[2 * kMaxSlabs + 1];
+    cudaError_t e = cudaEventRecord(ev_start, stream);
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(ctx->pipe_stream[i], ev_start, 0);
+    const int64_t per = (tiles + slabs - 1) / slabs;
+    for (int sidx = 0; sidx < slabs && e == cudaSuccess; ++sidx) {
+        const int64_t t0 = sidx * per, t1 = std::min<int64_t>(tiles, t0 + per);
+        if (t0 >= t1) break;
+        const int64_t c0 = t0 * ctx->sh.tile;
+        const int64_t c_in = ((t1 == tiles) ? ctx->ld : t1 * ctx->sh.tile) - c0;     // the last slab carries the padding
+        const int64_t c_out = std::min<int64_t>(ctx->N, t1 * ctx->sh.tile) - c0;
+        const float* src[4] = {x_host, delta_host, a_host, c_host};
+        float* dst[4] = {dev_x, dev_delta, dev_a, dev_c};
+        for (int k = 0; k < 4 && e == cudaSuccess; ++k)
+            e = cudaMemcpy2DAsync(dst[k] + c0, pitch, src[k] + c0, pitch, (size_t)c_in * sizeof(float),
+                                  (size_t)ctx->n, cudaMemcpyHostToDevice, s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->pipe_event[2 * sidx], s_in);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s_run, ctx->pipe_event[2 * sidx], 0);
+        if (e != cudaSuccess) break;
+        const ds_status st = run_step(ctx, dev_x, dev_delta, dev_a, dev_c, sigma, noise, hp, seed, step, s_run, t0, t1);
+        if (st != DS_OK) return st;
+        e = cudaEventRecord(ctx->pipe_event[2 * sidx + 1], s_run);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, ctx->pipe_event[2 * sidx + 1], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync(x_host + c0, pitch, dev_x + c0, pitch, (size_t)c_out * sizeof(float),
+                                  (size_t)ctx->n, cudaMemcpyDeviceToHost, s_out);
+        if (e == cudaSuccess)
+            e = cudaMemcpy2DAsync(delta_host + c0, pitch, dev_delta + c0, pitch, (size_t)c_out * sizeof(float),
+                                  (size_t)ctx->n, cudaMemcpyDeviceToHost, s_out);
+    }
+    // the caller's stream continues when the last slab is back (which implies every earlier stage)
+    if (e == cudaSuccess) e = cudaEventRecord(ev_done, s_out);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ev_done, 0);
     if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
     return DS_OK;
 }

@@ -425,7 +425,7 @@ __global__ void __launch_bounds__(1024, 1) ds_column_kernel(const __grid_constan
 
     const int64_t full_len = (int64_t)E * 32 * G;
     int buf = 0;
-    for (int64_t col = blockIdx.x; col < p.tiles; col += gridDim.x) {
+    for (int64_t col = p.tile_begin + blockIdx.x; col < p.tile_end; col += gridDim.x) {
         const int64_t remain = p.N - col * p.tile;
         const bool full = (p.tile == full_len) && (remain >= p.tile);
         if (full) column_body<CODE, NOISE, E, MODE, true>(p, L, smem, col, buf, lane, grp, wg, node, node_ok);

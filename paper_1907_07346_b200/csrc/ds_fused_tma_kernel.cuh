@@ -153,8 +153,8 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
         return true;
     };
 
-    int64_t col = blockIdx.x;
-    bool pending = (col < p.tiles) ? issue(col) : false;
+    int64_t col = p.tile_begin + blockIdx.x;
+    bool pending = (col < p.tile_end) ? issue(col) : false;
     // The gradient noise of a tile depends on nothing that is loaded, so it is
     // drawn one tile AHEAD (after the mixing of the previous tile): phase A then
     // only moves the slot into registers and takes the local step, and the refill
@@ -222,13 +222,13 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             }
         }
     };
-    if (col < p.tiles) draw_noise(col);      // (also when only the rounding stream is needed)
+    if (col < p.tile_end) draw_noise(col);      // (also when only the rounding stream is needed)
     uint32_t parity = 0;
     int buf = 0;
     constexpr float kL = (float)((1u << (T::kBits & 15)) - 1u);
     constexpr float kHalfL = 0.5f * kL;
 
-    for (; col < p.tiles; col += gridDim.x) {
+    for (; col < p.tile_end; col += gridDim.x) {
         const int64_t k0 = col * p.tile;
         const int64_t remain = p.N - k0;
         const int m_len = (int)(remain < p.tile ? remain : p.tile);
@@ -287,7 +287,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             __syncwarp();
             {
                 const int64_t next = col + gridDim.x;
-                pending = (next < p.tiles) ? issue(next) : false;
+                pending = (next < p.tile_end) ? issue(next) : false;
             }
 
             // ---- scale of the (node, tile) -----------------------------------
@@ -445,7 +445,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     st_partial(x_lane + 128 * r, make_float4(xa.x, xa.y, xb.x, xb.y), nv);
                 }
             }
-            if (col + gridDim.x < p.tiles) draw_noise(col + gridDim.x);
+            if (col + gridDim.x < p.tile_end) draw_noise(col + gridDim.x);
             return false;
         };
         const bool aborted = full ? tile_body(std::true_type{}) : tile_body(std::false_type{});

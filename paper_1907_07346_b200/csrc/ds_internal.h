@@ -29,6 +29,8 @@ struct StepParams {
     int32_t nnz;
     int64_t tile;             // elements per column tile (= chunk unless prescaled)
     int64_t tiles;            // column tiles per row
+    int64_t tile_begin;       // this launch covers the tiles [tile_begin, tile_end)
+    int64_t tile_end;
     const int32_t* row_ptr;   // device CSR of W - I
     const int32_t* col_idx;
     const float* wprime;      // W_ij - I_ij, binary32

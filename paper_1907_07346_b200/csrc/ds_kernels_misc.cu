@@ -1,5 +1,7 @@
 // Mix kernel of the two-kernel path, the per-node scale finaliser and the
 // random-stream diagnostic kernel.
+#include <algorithm>
+
 #include "ds_fused_tma_kernel.cuh"
 
 namespace ds {
@@ -19,9 +21,11 @@ __global__ void __launch_bounds__(256) ds_mix_kernel(const __grid_constant__ Ste
         __syncthreads();
     }
     const int node = blockIdx.y;
-    const int64_t nf4 = (p.N + 3) >> 2;
+    // this launch covers the tiles [tile_begin, tile_end): float4 indices [f_begin, f_end)
+    const int64_t f_begin = (p.tile_begin * p.tile) >> 2;
+    const int64_t nf4 = min((p.N + 3) >> 2, (p.tile_end * p.tile) >> 2);
     const int e_beg = p.row_ptr[node], e_end = p.row_ptr[node + 1];
-    for (int64_t f = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; f < nf4;
+    for (int64_t f = f_begin + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; f < nf4;
          f += (int64_t)gridDim.x * blockDim.x) {
         const int64_t k = 4 * f;
         const int nv = (int)min((int64_t)4, p.N - k);
@@ -67,9 +71,9 @@ __global__ void __launch_bounds__(256) ds_mix_kernel(const __grid_constant__ Ste
 }
 
 cudaError_t launch_mix_kernel(const StepParams& p, int code, cudaStream_t stream) {
-    const int64_t nf4 = (p.N + 3) >> 2;
+    const int64_t nf4 = std::min<int64_t>((p.N + 3) >> 2, (p.tile_end * p.tile) >> 2) - ((p.tile_begin * p.tile) >> 2);
     const int threads = 256;
-    int64_t bx = (nf4 + threads - 1) / threads;
+    int64_t bx = std::max<int64_t>(1, (nf4 + threads - 1) / threads);
     if (bx > 148 * 64) bx = 148 * 64;
     const dim3 grid((unsigned)bx, (unsigned)p.n);
     switch (code) {

@@ -91,6 +91,8 @@ extern "C" ds_status ds_node_scales_noalloc(float* scales_out, const float* x, c
     p.nnz = 0;
     p.tile = kTile;
     p.tiles = tiles;
+    p.tile_begin = 0;
+    p.tile_end = tiles;
     p.lut = reinterpret_cast<const float*>(scratch);          // the zero table
     p.partials = scratch + kTableSlots;
     p.scales = scales_out;

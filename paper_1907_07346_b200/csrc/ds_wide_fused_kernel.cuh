@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(512, 2) ds_wide_fused_kernel(const __grid_cons
 
     const int64_t full_len = (int64_t)E * 32 * G;
     int buf = 0, red_parity = 0;
-    for (int64_t col = blockIdx.x; col < p.tiles; col += gridDim.x) {
+    for (int64_t col = p.tile_begin + blockIdx.x; col < p.tile_end; col += gridDim.x) {
         const int64_t remain = p.N - col * p.tile;
         const bool full = (p.tile == full_len) && (remain >= p.tile);
         if (full) wide_column<CODE, NOISE, E, true>(p, L, smem, col, buf, red_parity, lane, grp, wg);

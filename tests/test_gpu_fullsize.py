@@ -77,3 +77,42 @@ def test_full_size_windows(name, N):
             assert _rel(gx[:, k0:k0 + cols], st[0]) <= TOL, (name, t, k0)
             assert _rel(gd[:, k0:k0 + cols], st[1]) <= TOL, (name, t, k0)
     ds.close()
+
+
+def test_host_buffer_entry_point_pipelined():
+    """ds_step_host on arrays large enough (>= 64 MiB each) to take the slab
+    pipeline (copies in, compute and copies out overlapped on internal streams):
+    same result as the oracle, padding columns never written back."""
+    import torch
+    from oracle import oracle as orc
+    from paper_1907_07346_b200 import binding as B
+    g = I.ring(8)
+    N = 512 * 4200 + 40
+    ld = I.row_pitch(N) + 32
+    rng = np.random.default_rng(5)
+    host = []
+    for scale in (0.3, 0.05, None, 1.0):
+        arr = np.full((g.n, ld), 3.0, np.float32)
+        if scale is None:
+            arr[:, :N] = rng.random((g.n, N), dtype=np.float32) * np.float32(1.5) + np.float32(0.5)
+        else:
+            arr[:, :N] = rng.standard_normal((g.n, N), dtype=np.float32) * np.float32(scale)
+        host.append(arr)
+    assert host[0].nbytes >= 64 << 20
+    ds = B.DeepSqueeze(g, N, ld, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512)
+    pinned = [torch.from_numpy(h.copy()).pin_memory() for h in host]
+    dev = [torch.empty((g.n, ld), dtype=torch.float32, device="cuda") for _ in range(4)]
+    side = torch.cuda.Stream()
+    for t in range(2):
+        ds.ds_step_host(pinned[0], pinned[1], pinned[2], pinned[3], 0.1, I.NOISE_GAUSS, 0.01, 0.5, 9, t,
+                        *dev, stream=side)
+    ds.ds_sync(side)
+    for t in range(2):
+        codes_ref, scales_ref, _, _ = orc.step(g, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, host[0], host[1],
+                                               host[2], host[3], N, 0.1, I.NOISE_GAUSS, 0.01, 0.5, 9, t)
+    codes, scales = ds.codes_to_host()
+    assert np.array_equal(codes, codes_ref)
+    assert _rel(pinned[0].numpy()[:, :N], host[0][:, :N]) <= TOL
+    assert _rel(pinned[1].numpy()[:, :N], host[1][:, :N]) <= TOL
+    assert np.all(pinned[0].numpy()[:, N:] == 3.0) and np.all(pinned[1].numpy()[:, N:] == 3.0)
+    ds.close()
