@@ -119,8 +119,10 @@ typedef struct {
  *                      x - gamma g in registers and the column's C[v] in shared memory, and
  *                      mixes without re-reading anything from global memory.  Where the
  *                      column fits in shared memory this is the persistent kernel whose
- *                      inputs are staged by bulk asynchronous copies (TMA); otherwise the
- *                      variant below.
+ *                      inputs are staged by bulk asynchronous copies (TMA); for columns of
+ *                      many nodes or long chunks the same kernel sweeps the nodes in batches
+ *                      (x - gamma g parked in x and re-read from L2, packed codes of the whole
+ *                      column in shared memory); otherwise the variant below.
  *   DS_PATH_FUSED_LDG  the fused kernel with direct vector loads and packed codes in shared
  *                      memory (one block per column).  When a block cannot hold all nodes of
  *                      a column at once (many nodes, long chunks) it sweeps them in batches:

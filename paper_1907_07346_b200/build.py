@@ -17,9 +17,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdeepsqueeze.so")
-SOURCES = ["ds_api.cu", "ds_kernels_tma.cu", "ds_kernels_fused.cu", "ds_kernels_wide.cu", "ds_kernels_compress.cu",
+SOURCES = ["ds_api.cu", "ds_kernels_tma.cu", "ds_kernels_fused.cu", "ds_kernels_wide.cu", "ds_kernels_wide_tma.cu", "ds_kernels_compress.cu",
            "ds_kernels_misc.cu", "ds_noalloc.cu"]
-HEADERS = ["ds_device.cuh", "ds_internal.h", "ds_column_kernel.cuh", "ds_fused_tma_kernel.cuh", "ds_wide_fused_kernel.cuh"]
+HEADERS = ["ds_device.cuh", "ds_internal.h", "ds_column_kernel.cuh", "ds_fused_tma_kernel.cuh", "ds_wide_fused_kernel.cuh", "ds_wide_tma_kernel.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-fmad=false", "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
 

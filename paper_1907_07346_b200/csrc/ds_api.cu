@@ -9,6 +9,7 @@
 #include "../../include/deepsqueeze.h"
 #include "ds_fused_tma_kernel.cuh"
 #include "ds_wide_fused_kernel.cuh"
+#include "ds_wide_tma_kernel.cuh"
 
 using namespace ds;
 
@@ -173,6 +174,25 @@ Plan plan_wide(const Shape& sh, int32_t n, int32_t nnz, int force_e = 0) {
     return pl;
 }
 
+// Persistent TMA-staged kernel that sweeps the nodes of a column in batches.
+Plan plan_wide_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int force_e = 0) {
+    Plan pl;
+    int E, G;
+    pick_lane_shape(sh.tile, force_e, &E, &G);
+    pl.elems_per_lane = E;
+    pl.warps_per_group = G;
+    if (sh.code == CODE_ID32 || sh.code == CODE_N2 || sh.code == CODE_N4 || E < 8 || G > 16 || num_sms < 1) return pl;
+    const int npb = std::max(1, std::min<int>(n, 16 / G));
+    pl.nodes_per_block = npb;
+    pl.block = dim3((unsigned)(npb * G * 32));
+    const bool lut = (sh.code != CODE_SIGN);
+    pl.smem = wide_tma_smem_layout(sh.code_bits, lut, E, npb * G, sh.tile, n, nnz).total;
+    if (pl.smem > (size_t)kMaxSmem) return pl;
+    pl.grid = dim3((unsigned)std::min<int64_t>(sh.tiles, num_sms));
+    pl.ok = true;
+    return pl;
+}
+
 }  // namespace
 
 struct ds_ctx {
@@ -183,7 +203,7 @@ struct ds_ctx {
     WsLayout ws;
     unsigned char* base;
     int path_req;
-    Plan tma, fused, wide, compress, reduce;
+    Plan tma, wide_tma, fused, wide, compress, reduce;
     int num_sms;
     bool pipe_ready;                                  // streams / events of ds_step_host
     cudaStream_t pipe_stream[3];
@@ -292,6 +312,7 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     }
     ctx->num_sms = sms;
     ctx->tma = plan_tma(sh, n, nnz, sms);
+    ctx->wide_tma = plan_wide_tma(sh, n, nnz, sms);
     ctx->fused = plan_column(MODE_FUSED, sh, n, nnz);
     ctx->wide = plan_wide(sh, n, nnz);
 
@@ -331,11 +352,14 @@ void ds_destroy(ds_ctx* ctx) {
     delete ctx;
 }
 
-// 2: persistent TMA-staged fused kernel, 1: fused kernel with direct loads,
-// 3: the same in node batches (wide columns), 0: two kernels
+// 2: persistent TMA-staged fused kernel, 4: the same with the nodes in batches,
+// 1: fused kernel with direct loads, 3: the same in node batches, 0: two kernels
 static int fused_kind(const ds_ctx* ctx) {
     if (ctx->path_req == DS_PATH_SPLIT) return 0;
-    if (ctx->path_req != DS_PATH_FUSED_LDG && ctx->tma.ok) return 2;
+    if (ctx->path_req != DS_PATH_FUSED_LDG) {
+        if (ctx->tma.ok) return 2;
+        if (ctx->wide_tma.ok) return 4;
+    }
     if (ctx->fused.ok) return 1;
     return ctx->wide.ok ? 3 : 0;
 }
@@ -343,7 +367,8 @@ static int fused_kind(const ds_ctx* ctx) {
 ds_status ds_set_path(ds_ctx* ctx, int32_t path) {
     if (!ctx) return DS_ERR_NULL;
     if (path < DS_PATH_AUTO || path > DS_PATH_FUSED_LDG) return DS_ERR_ARG;
-    if (path == DS_PATH_FUSED && !ctx->fused.ok && !ctx->tma.ok && !ctx->wide.ok) return DS_ERR_UNSUPPORTED;
+    if (path == DS_PATH_FUSED && !ctx->fused.ok && !ctx->tma.ok && !ctx->wide.ok && !ctx->wide_tma.ok)
+        return DS_ERR_UNSUPPORTED;
     if (path == DS_PATH_FUSED_LDG && !ctx->fused.ok && !ctx->wide.ok) return DS_ERR_UNSUPPORTED;
     ctx->path_req = path;
     return DS_OK;
@@ -358,6 +383,7 @@ ds_status ds_tune(ds_ctx* ctx, int32_t elems_per_lane) {
     ctx->compress = compress;
     ctx->reduce = plan_column(MODE_REDUCE, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
     ctx->tma = plan_tma(ctx->sh, ctx->n, ctx->nnz, ctx->num_sms, elems_per_lane);
+    ctx->wide_tma = plan_wide_tma(ctx->sh, ctx->n, ctx->nnz, ctx->num_sms, elems_per_lane);
     ctx->fused = plan_column(MODE_FUSED, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
     ctx->wide = plan_wide(ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
     return DS_OK;
@@ -367,9 +393,10 @@ ds_status ds_get_info(const ds_ctx* ctx, ds_info* info) {
     if (!ctx || !info) return DS_ERR_NULL;
     const int kind = fused_kind(ctx);
     const bool fused = kind != 0;
-    const Plan& pl = (kind == 2) ? ctx->tma : (kind == 1) ? ctx->fused : (kind == 3) ? ctx->wide : ctx->compress;
-    info->path = (kind == 2) ? DS_PATH_FUSED : (kind != 0) ? DS_PATH_FUSED_LDG : DS_PATH_SPLIT;
-    info->node_batches = (kind == 3) ? (ctx->n + pl.nodes_per_block - 1) / pl.nodes_per_block : 1;
+    const Plan& pl = (kind == 2) ? ctx->tma : (kind == 4) ? ctx->wide_tma : (kind == 1) ? ctx->fused
+                   : (kind == 3) ? ctx->wide : ctx->compress;
+    info->path = (kind == 2 || kind == 4) ? DS_PATH_FUSED : (kind != 0) ? DS_PATH_FUSED_LDG : DS_PATH_SPLIT;
+    info->node_batches = (kind == 3 || kind == 4) ? (ctx->n + pl.nodes_per_block - 1) / pl.nodes_per_block : 1;
     info->launches_per_step = (fused ? 1 : 2) + (ctx->sh.per_node ? 2 : 0);
     info->elems_per_lane = pl.elems_per_lane;
     info->warps_per_chunk = pl.warps_per_group;
@@ -445,6 +472,10 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
             p.warps_per_group = ctx->tma.warps_per_group;
             p.nodes_per_block = ctx->tma.nodes_per_block;
             e = launch_fused_tma(shape_of(ctx->tma, MODE_FUSED), p, stream);
+        } else if (kind == 4) {
+            p.warps_per_group = ctx->wide_tma.warps_per_group;
+            p.nodes_per_block = ctx->wide_tma.nodes_per_block;
+            e = launch_fused_wide_tma(shape_of(ctx->wide_tma, MODE_FUSED), p, stream);
         } else if (kind == 3) {
             p.warps_per_group = ctx->wide.warps_per_group;
             p.nodes_per_block = ctx->wide.nodes_per_block;

@@ -65,6 +65,7 @@ struct LaunchShape {
 // Launchers (defined in the kernel translation units).
 cudaError_t launch_column_fused(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_fused_tma(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
+cudaError_t launch_fused_wide_tma(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_fused_wide(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_column_compress(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_column_reduce(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);

@@ -409,7 +409,7 @@ def test_results_do_not_depend_on_tuning_or_stream(env):
             assert np.array_equal(u, v)
 
 
-@pytest.mark.parametrize("path", [3, 2])
+@pytest.mark.parametrize("path", [1, 3, 2])
 def test_many_nodes(env, path):
     """200 nodes on a ring: far more than one block holds (node batches on the
     wide kernel, many grid rows on the two-kernel path)."""
