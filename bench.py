@@ -51,8 +51,8 @@ def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) ->
 # profiles/ds_fused_tma_kernel_cfg3_small_counters.md (dram__bytes_read.sum +
 # dram__bytes_write.sum over one launch of 67,108,864 updates), valid for the
 # kernel sources whose digest is recorded beside it.
-NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59403e9 / 67108864,
-               "sources_sha256": "2a0e63f6a985c443068057d1262668a39d7739850ef37c0b429b36459aad161a"}
+NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59429e9 / 67108864,
+               "sources_sha256": "77e7338c5659be51fb15218266c863c8bb88b2d0824e8dc8284b04ef259eb4f0"}
 KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
 
 
