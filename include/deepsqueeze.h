@@ -187,6 +187,23 @@ ds_status ds_step(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
 ds_status ds_step_g(ds_ctx *ctx, float *x, float *delta, const float *g, const ds_hparams *hp,
                     uint64_t seed, uint64_t step, void *cuda_stream);
 
+/* T consecutive iterations t = step0 .. step0+T-1 of Algorithm 1 with a
+ * per-iteration schedule (Section 5 decays the learning rate): iteration t uses
+ * gamma = gammas[t-step0] and eta = etas[t-step0].  The launches of all T
+ * iterations are recorded once into a CUDA graph (captured on an internal
+ * stream, nothing runs during capture) and replayed on `cuda_stream` as one
+ * submission, which removes the per-launch host cost that bounds small
+ * problems.  The executable graph is kept in the context: a later call with
+ * the same T updates its kernel arguments in place instead of instantiating
+ * again.  Results are bit-identical to T calls of ds_step.
+ *   gammas, etas  host arrays of T binary32 values, read before the call returns
+ *   T             1 .. DS_RUN_MAX_STEPS
+ * Errors: as ds_step; DS_ERR_ARG if T is out of range or step0 + T > 2^56. */
+#define DS_RUN_MAX_STEPS 4096
+ds_status ds_run(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
+                 const float *gammas, const float *etas, int32_t T,
+                 uint64_t seed, uint64_t step0, void *cuda_stream);
+
 /* Same iteration for HOST buffers: x, delta, a, c (host, [n][ld]) go to the
  * caller's device staging arrays, the step runs, and x and delta come back,
  * all ordered after the work already in `cuda_stream`; that stream continues

@@ -208,6 +208,9 @@ struct ds_ctx {
     bool pipe_ready;                                  // streams / events of ds_step_host
     cudaStream_t pipe_stream[3];
     cudaEvent_t pipe_event[2 * kMaxSlabs + 2];
+    cudaStream_t capture_stream;                      // ds_run records its graph here
+    cudaGraphExec_t run_exec;                         // executable graph of the last ds_run
+    int32_t run_exec_steps;                           // T it was instantiated for (0 = none)
 };
 
 extern "C" {
@@ -300,6 +303,9 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     ctx->base = static_cast<unsigned char*>(workspace);
     ctx->path_req = DS_PATH_AUTO;
     ctx->pipe_ready = false;
+    ctx->capture_stream = nullptr;
+    ctx->run_exec = nullptr;
+    ctx->run_exec_steps = 0;
     ctx->compress = plan_column(MODE_COMPRESS, sh, n, nnz);
     ctx->reduce = plan_column(MODE_REDUCE, sh, n, nnz);
     if (!ctx->compress.ok) { delete ctx; return DS_ERR_UNSUPPORTED; }
@@ -345,6 +351,9 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
 
 void ds_destroy(ds_ctx* ctx) {
     if (!ctx) return;
+    // an executable graph still in flight is freed by the runtime once it completes
+    if (ctx->run_exec) (void)cudaGraphExecDestroy(ctx->run_exec);
+    if (ctx->capture_stream) (void)cudaStreamDestroy(ctx->capture_stream);
     if (ctx->pipe_ready) {
         for (int i = 0; i < 3; ++i) (void)cudaStreamDestroy(ctx->pipe_stream[i]);
         for (int i = 0; i < 2 * kMaxSlabs + 2; ++i) (void)cudaEventDestroy(ctx->pipe_event[i]);
@@ -509,6 +518,71 @@ ds_status ds_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, const d
                     uint64_t seed, uint64_t step, void* cuda_stream) {
     if (!ctx || !x || !delta || !g || !hp) return DS_ERR_NULL;
     return run_step(ctx, x, delta, g, nullptr, 0.0f, GRAD_GIVEN, hp, seed, step, cuda_stream);
+}
+
+ds_status ds_run(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const float* gammas,
+                 const float* etas, int32_t T, uint64_t seed, uint64_t step0, void* cuda_stream) {
+    if (!ctx || !x || !delta || !gp || !gp->a || !gp->c || !gammas || !etas) return DS_ERR_NULL;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    if (T < 1 || T > DS_RUN_MAX_STEPS) return DS_ERR_ARG;
+    if (step0 >= ((uint64_t)1 << 56) || step0 + (uint64_t)T > ((uint64_t)1 << 56)) return DS_ERR_ARG;
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
+                           reinterpret_cast<uintptr_t>(gp->a) | reinterpret_cast<uintptr_t>(gp->c);
+    if ((bits % 16) != 0) return DS_ERR_ALIGN;
+    if (!ctx->capture_stream &&
+        cudaStreamCreateWithFlags(&ctx->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        (void)cudaGetLastError();
+        ctx->capture_stream = nullptr;
+        return DS_ERR_CUDA;
+    }
+    // Record: the launches go into a graph, none of them runs here.
+    if (cudaStreamBeginCapture(ctx->capture_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DS_ERR_CUDA;
+    }
+    ds_status st = DS_OK;
+    for (int32_t t = 0; t < T && st == DS_OK; ++t) {
+        const ds_hparams hp = {gammas[t], etas[t]};
+        st = run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, gp->noise, &hp, seed, step0 + (uint64_t)t,
+                      ctx->capture_stream);
+    }
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamEndCapture(ctx->capture_stream, &graph);    // always ends the capture
+    if (st != DS_OK || e != cudaSuccess || !graph) {
+        (void)cudaGetLastError();
+        if (graph) (void)cudaGraphDestroy(graph);
+        return st != DS_OK ? st : DS_ERR_CUDA;
+    }
+    // Same T as last time: same topology, only kernel arguments differ.
+    if (ctx->run_exec && ctx->run_exec_steps == T) {
+        cudaGraphExecUpdateResultInfo info;
+        if (cudaGraphExecUpdate(ctx->run_exec, graph, &info) != cudaSuccess) {
+            (void)cudaGetLastError();
+            (void)cudaGraphExecDestroy(ctx->run_exec);
+            ctx->run_exec = nullptr;
+        }
+    } else if (ctx->run_exec) {
+        (void)cudaGraphExecDestroy(ctx->run_exec);
+        ctx->run_exec = nullptr;
+    }
+    if (!ctx->run_exec) {
+        ctx->run_exec_steps = 0;
+        e = cudaGraphInstantiate(&ctx->run_exec, graph, 0);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            ctx->run_exec = nullptr;
+            (void)cudaGraphDestroy(graph);
+            return DS_ERR_CUDA;
+        }
+        ctx->run_exec_steps = T;
+    }
+    (void)cudaGraphDestroy(graph);
+    e = cudaGraphLaunch(ctx->run_exec, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DS_ERR_CUDA;
+    }
+    return DS_OK;
 }
 
 // Streams and events of the host-buffer entry point, made on first use.

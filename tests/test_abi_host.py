@@ -161,6 +161,7 @@ def test_null_handles():
     L = B.lib()
     assert L.ds_step(None, None, None, None, None, 0, 0, None) == B.DS_ERR_NULL
     assert L.ds_step_g(None, None, None, None, None, 0, 0, None) == B.DS_ERR_NULL
+    assert L.ds_run(None, None, None, None, None, None, 1, 0, 0, None) == B.DS_ERR_NULL
     assert L.ds_set_path(None, 0) == B.DS_ERR_NULL
     assert L.ds_get_info(None, None) == B.DS_ERR_NULL
     assert L.ds_codes(None, None, None, None, None) == B.DS_ERR_NULL
