@@ -25,6 +25,9 @@
  * build with -ffp-contract=off so the compiler adds no fusion of its own.
  * Scale sums are accumulated in binary64.
  *
+ * oracle_ecsgd_step() is the centralized error-compensated SGD of Section 1
+ * (a baseline that shares the compressors), stated the same way.
+ *
  * Parity pins: see tests/test_oracle_*.py (compression identity, mean
  * preservation, dense float64 matrix form, D-PSGD closed form, gradient
  * descent closed form, hand-worked golden cases, exhaustive accuracy of the
@@ -454,6 +457,88 @@ int oracle_step(int32_t n, int64_t N, int64_t ld,
     }
     if (C_out) memcpy(C_out, C, sizeof(float) * (size_t)n * (size_t)N);
     free(h); free(C);
+    return 0;
+}
+
+/*
+ * Centralized error-compensated SGD, the scheme the paper starts from
+ * (Section 1, the three displayed updates) and one of its baselines:
+ *     g'    <- C[g + delta]                 on each worker
+ *     delta <- (g + delta) - C[g + delta]   on each worker
+ *     x     <- x - gamma g'                 on the server
+ * The paper writes it for one worker.  Reading for n workers: row i of x is
+ * worker i's copy of the model, worker i evaluates its own objective there, and
+ * the server's average is the weighted sum over the rows of W (complete graph
+ * with W_ij = 1/n = the parameter server; then all rows stay equal):
+ *     g  = fma(a, d, sigma z)  (or the given gradient)
+ *     v  = g + delta
+ *     (C, code) = compress(v) per chunk ;  delta' = v - C
+ *     acc = 0; for j in N(i) ascending: acc = fma(W_ij, C_j, acc)
+ *     x'  = fma(-gamma, acc, x)
+ * Random streams, compressors, chunking and packing are those of oracle_step.
+ */
+int oracle_ecsgd_step(int32_t n, int64_t N, int64_t ld,
+                      const int32_t *row_ptr, const int32_t *col_idx, const float *W,
+                      int comp_kind, int bits, int64_t chunk,
+                      float *x, float *delta, const float *a, const float *c,
+                      float sigma, int noise_kind, float gamma,
+                      uint64_t seed, uint64_t step,
+                      uint32_t *codes, int64_t code_pitch,
+                      float *scales, int64_t scales_pitch, const float *g_given)
+{
+    if (chunk <= 0) chunk = N;
+    int code_bits = (comp_kind == COMP_IDENTITY) ? 32
+                  : (comp_kind == COMP_SIGN1_L1) ? 1 : bits;
+    int64_t M = (N + chunk - 1) / chunk;
+    int64_t words = (N * (int64_t)code_bits + 31) / 32;
+    float *C = (float *)malloc(sizeof(float) * (size_t)n * (size_t)N);
+    float *v = (float *)malloc(sizeof(float) * (size_t)chunk);
+    float *r = (float *)malloc(sizeof(float) * (size_t)chunk);
+    uint32_t *q = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)chunk);
+    if (!C || !v || !r || !q) { free(C); free(v); free(r); free(q); return -1; }
+
+    /* workers */
+    for (int32_t i = 0; i < n; ++i) {
+        memset(codes + (size_t)i * code_pitch, 0, sizeof(uint32_t) * (size_t)words);
+        for (int64_t mi = 0; mi < M; ++mi) {
+            int64_t k0 = mi * chunk;
+            int64_t m = (N - k0 < chunk) ? (N - k0) : chunk;
+            for (int64_t kk = 0; kk < m; ++kk) {
+                int64_t k = k0 + kk;
+                size_t at = (size_t)i * (size_t)ld + (size_t)k;
+                float g;
+                if (g_given) {
+                    g = g_given[at];
+                } else {
+                    float z = oracle_noise_elem(noise_kind, seed, (uint32_t)i, step, k);
+                    float d = x[at] - c[at];
+                    float nz = sigma * z;
+                    g = fmaf(a[at], d, nz);
+                }
+                v[kk] = g + delta[at];
+                r[kk] = (comp_kind == COMP_UNIFORM_STOCH_MAXABS)
+                            ? oracle_rnd24_elem(seed, (uint32_t)i, step, k) : 0.0f;
+            }
+            float s;
+            float *Crow = C + (size_t)i * (size_t)N + (size_t)k0;
+            oracle_compress_chunk(comp_kind, bits, v, m, r, &s, q, Crow);
+            scales[(size_t)i * (size_t)scales_pitch + (size_t)mi] = s;
+            for (int64_t kk = 0; kk < m; ++kk)
+                delta[(size_t)i * (size_t)ld + (size_t)(k0 + kk)] = v[kk] - Crow[kk];
+            oracle_pack_codes(code_bits, q, k0, m, codes + (size_t)i * code_pitch);
+        }
+    }
+    /* server */
+    for (int32_t i = 0; i < n; ++i) {
+        for (int64_t k = 0; k < N; ++k) {
+            float acc = 0.0f;
+            for (int32_t e = row_ptr[i]; e < row_ptr[i + 1]; ++e)
+                acc = fmaf(W[e], C[(size_t)col_idx[e] * (size_t)N + (size_t)k], acc);
+            size_t at = (size_t)i * (size_t)ld + (size_t)k;
+            x[at] = fmaf(-gamma, acc, x[at]);
+        }
+    }
+    free(C); free(v); free(r); free(q);
     return 0;
 }
 

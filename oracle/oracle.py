@@ -51,6 +51,14 @@ def lib():
             C.c_uint64, C.c_uint64,
             _u32p, C.c_int64, _f32p, C.c_int64, _f32p, _f32p, C.c_int64, _f32p]
         L.oracle_step.restype = C.c_int
+        L.oracle_ecsgd_step.argtypes = [
+            C.c_int32, C.c_int64, C.c_int64, _i32p, _i32p, _f32p,
+            C.c_int, C.c_int, C.c_int64,
+            _f32p, _f32p, _f32p, _f32p,
+            C.c_float, C.c_int, C.c_float,
+            C.c_uint64, C.c_uint64,
+            _u32p, C.c_int64, _f32p, C.c_int64, _f32p]
+        L.oracle_ecsgd_step.restype = C.c_int
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = C.c_int
         _lib = L
@@ -159,6 +167,36 @@ def step(graph, comp_kind: int, bits: int, chunk: int, x: np.ndarray, delta: np.
     if rc != 0:
         raise MemoryError("oracle_step could not allocate")
     return codes, scales, v, Cv
+
+
+def ecsgd_step(graph, comp_kind: int, bits: int, chunk: int, x: np.ndarray, delta: np.ndarray,
+               a: np.ndarray, c: np.ndarray, N: int, sigma: float, noise_kind: int,
+               gamma: float, seed: int, step_index: int, g_given: np.ndarray | None = None):
+    """One iteration of centralized error-compensated SGD (Section 1) in place
+    on x, delta ([n][ld] float32): row i is worker i's copy of the model, the
+    server's average uses row i of W.  Returns (codes, scales)."""
+    n, ld = x.shape
+    for arr in (x, delta, a, c) + (() if g_given is None else (g_given,)):
+        assert arr.dtype == np.float32 and arr.flags.c_contiguous and arr.shape == (n, ld)
+    assert graph.n == n and N <= ld
+    cb = code_bits(comp_kind, bits)
+    words = (N * cb + 31) // 32
+    ch = chunk if chunk > 0 else N
+    M = (N + ch - 1) // ch
+    codes = np.zeros((n, words), dtype=np.uint32)
+    scales = np.zeros((n, M), dtype=np.float32)
+    rp = np.ascontiguousarray(graph.row_ptr, dtype=np.int32)
+    ci = np.ascontiguousarray(graph.col_idx, dtype=np.int32)
+    w = np.ascontiguousarray(graph.w, dtype=np.float32)
+    rc = lib().oracle_ecsgd_step(
+        n, N, ld, _p(rp, _i32p), _p(ci, _i32p), _p(w, _f32p), comp_kind, bits, chunk,
+        _p(x, _f32p), _p(delta, _f32p), _p(a, _f32p), _p(c, _f32p),
+        sigma, noise_kind, gamma, seed, step_index,
+        _p(codes, _u32p), words, _p(scales, _f32p), M,
+        None if g_given is None else _p(g_given, _f32p))
+    if rc != 0:
+        raise MemoryError("oracle_ecsgd_step could not allocate")
+    return codes, scales
 
 
 def num_threads() -> int:

@@ -68,6 +68,14 @@ def ring(n: int) -> Graph:
                                 f"ring{n}")
 
 
+def complete(n: int) -> Graph:
+    """Complete graph with W_ij = 1/n: every node averages all nodes (the
+    parameter server of centralized training)."""
+    if n < 1:
+        raise ValueError("n >= 1")
+    return _from_neighbour_sets([set(range(n)) - {i} for i in range(n)], f"complete{n}")
+
+
 def torus(rows: int, cols: int) -> Graph:
     """2-D torus rows x cols: four neighbours (up, down, left, right, wrapped)."""
     if rows < 3 or cols < 3:
