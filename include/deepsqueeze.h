@@ -187,6 +187,28 @@ ds_status ds_step(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
 ds_status ds_step_g(ds_ctx *ctx, float *x, float *delta, const float *g, const ds_hparams *hp,
                     uint64_t seed, uint64_t step, void *cuda_stream);
 
+/* One iteration of CENTRALIZED error-compensated SGD (Section 1, the three
+ * displayed updates; one of the baselines of Section 5), on the same state
+ * layout and with the same compressors, chunking, packing and random streams:
+ *     workers:  v_i = g_i + delta_i;  C[v_i];  delta_i <- v_i - C[v_i]
+ *     server:   x_i <- x_i - gamma sum_{j in N(i)} W_ij C[v_j]
+ * The paper writes it for one worker.  Here row i of x is worker i's copy of
+ * the model, and the server's average is the weighted sum over row i of W: a
+ * complete graph with W_ij = 1/n is the parameter server (all rows of x then
+ * stay equal if they start equal).  Operation order per element:
+ *     d = x - c; g = fma(a, d, sigma z); v = g + delta; compress; delta' = v - C;
+ *     acc = 0; for j in N(i) ascending: acc = fma(W_ij, C_j, acc); x' = fma(-gamma, acc, x).
+ * Always two kernels (the workers' compression, then the server's update, which
+ * streams each worker's packed codes once); ds_set_path has no effect on it.
+ * Traffic: 24 + b/8 + 4/chunk bytes per node-element plus the codes re-read by
+ * the server ((deg+1) b/8, served by L2 where the codes fit).
+ * Arguments and errors as ds_step / ds_step_g; ds_codes returns what the
+ * workers sent. */
+ds_status ds_ecsgd_step(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
+                        float gamma, uint64_t seed, uint64_t step, void *cuda_stream);
+ds_status ds_ecsgd_step_g(ds_ctx *ctx, float *x, float *delta, const float *g,
+                          float gamma, uint64_t seed, uint64_t step, void *cuda_stream);
+
 /* T consecutive iterations t = step0 .. step0+T-1 of Algorithm 1 with a
  * per-iteration schedule (Section 5 decays the learning rate): iteration t uses
  * gamma = gammas[t-step0] and eta = etas[t-step0].  The launches of all T

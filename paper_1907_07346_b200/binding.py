@@ -24,7 +24,7 @@ DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 DS_RUN_MAX_STEPS = 4096
 
-EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_g", "ds_run", "ds_step_host", "ds_codes", "ds_set_path",
+EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_g", "ds_ecsgd_step", "ds_ecsgd_step_g", "ds_run", "ds_step_host", "ds_codes", "ds_set_path",
            "ds_tune", "ds_get_info", "ds_sync", "ds_selftest_timeout", "ds_selftest_math", "ds_noise", "ds_node_scales_noalloc",
            "ds_destroy", "ds_strerror"]
 
@@ -73,6 +73,12 @@ def lib():
         L.ds_step_g.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ds_hparams),
                                 C.c_uint64, C.c_uint64, C.c_void_p]
         L.ds_step_g.restype = C.c_int
+        L.ds_ecsgd_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ds_grad_params), C.c_float,
+                                    C.c_uint64, C.c_uint64, C.c_void_p]
+        L.ds_ecsgd_step.restype = C.c_int
+        L.ds_ecsgd_step_g.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
+                                      C.c_uint64, C.c_uint64, C.c_void_p]
+        L.ds_ecsgd_step_g.restype = C.c_int
         L.ds_run.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ds_grad_params), C.POINTER(C.c_float),
                              C.POINTER(C.c_float), C.c_int32, C.c_uint64, C.c_uint64, C.c_void_p]
         L.ds_run.restype = C.c_int
@@ -216,6 +222,26 @@ class DeepSqueeze:
         s = torch.cuda.current_stream(self.device) if stream is None else stream
         _check(lib().ds_step_g(self.ctx, x.data_ptr(), delta.data_ptr(), g.data_ptr(), C.byref(hp),
                                seed, step, C.c_void_p(s.cuda_stream)), "ds_step_g")
+
+    def ds_ecsgd_step(self, x, delta, a, c, sigma: float, noise: int, gamma: float, seed: int, step: int,
+                      stream=None):
+        """One iteration of centralized error-compensated SGD in place on x, delta."""
+        torch = self.torch
+        for t in (x, delta, a, c):
+            assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (self.n, self.ld)
+        gp = ds_grad_params(a.data_ptr(), c.data_ptr(), sigma, noise)
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        _check(lib().ds_ecsgd_step(self.ctx, x.data_ptr(), delta.data_ptr(), C.byref(gp), gamma,
+                                   seed, step, C.c_void_p(s.cuda_stream)), "ds_ecsgd_step")
+
+    def ds_ecsgd_step_g(self, x, delta, g, gamma: float, seed: int, step: int, stream=None):
+        """The same iteration with the gradient supplied as a device tensor g[n][ld]."""
+        torch = self.torch
+        for t in (x, delta, g):
+            assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (self.n, self.ld)
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        _check(lib().ds_ecsgd_step_g(self.ctx, x.data_ptr(), delta.data_ptr(), g.data_ptr(), gamma,
+                                     seed, step, C.c_void_p(s.cuda_stream)), "ds_ecsgd_step_g")
 
     def ds_step_host(self, x_h, delta_h, a_h, c_h, sigma, noise, gamma, eta, seed, step,
                      dev_x, dev_delta, dev_a, dev_c, stream=None):

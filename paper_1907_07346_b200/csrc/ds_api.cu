@@ -35,7 +35,7 @@ struct Shape {
 };
 
 struct WsLayout {
-    size_t codes, scales, dscales, partials, row_ptr, col_idx, wprime, lut, error_flag, total;
+    size_t codes, scales, dscales, partials, row_ptr, col_idx, wprime, wplain, lut, error_flag, total;
 };
 
 bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
@@ -88,6 +88,7 @@ WsLayout make_ws(int32_t n, int32_t nnz, const Shape& sh) {
     w.row_ptr = off;  off = align_up(off + (size_t)(n + 1) * 4, kAlign);
     w.col_idx = off;  off = align_up(off + (size_t)nnz * 4, kAlign);
     w.wprime = off;   off = align_up(off + (size_t)nnz * 4, kAlign);
+    w.wplain = off;   off = align_up(off + (size_t)nnz * 4, kAlign);
     w.lut = off;      off = align_up(off + 256 * 4, kAlign);
     w.error_flag = off; off = align_up(off + 4, kAlign);
     w.total = off;
@@ -336,6 +337,7 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     cudaError_t e = cudaMemcpy(ctx->base + ws.row_ptr, rp, (size_t)(n + 1) * 4, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.col_idx, ci, (size_t)nnz * 4, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.wprime, wprime.data(), (size_t)nnz * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.wplain, W, (size_t)nnz * 4, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(ctx->base + ws.lut, lut, sizeof(lut), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.codes, 0, ws.scales - ws.codes);
     if (e == cudaSuccess) e = cudaMemset(ctx->base + ws.scales, 0, ws.partials - ws.scales);   // scales and decode factors
@@ -428,9 +430,14 @@ ds_status ds_codes(ds_ctx* ctx, const uint32_t** codes, int64_t* code_pitch_word
 
 // One iteration; `grad_kind` is a NOISE_* value for the synthetic gradient
 // (a, c given) or GRAD_GIVEN (a is the gradient itself, c unused).
+// ecsgd: the iteration of centralized error-compensated SGD (Section 1) instead
+// of Algorithm 1 -- always two kernels: the workers' compression of g + delta,
+// then the server's x <- x - gamma sum_j W_ij C_j, which is the mix kernel run
+// with the weights W themselves and -gamma in the place of eta.
 static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, const float* c,
                           float sigma, int grad_kind, const ds_hparams* hp, uint64_t seed,
-                          uint64_t step, void* cuda_stream, int64_t tile_begin = 0, int64_t tile_end = -1) {
+                          uint64_t step, void* cuda_stream, int64_t tile_begin = 0, int64_t tile_end = -1,
+                          bool ecsgd = false) {
     if (step >= ((uint64_t)1 << 56)) return DS_ERR_ARG;
     if (tile_end < 0) tile_end = ctx->sh.tiles;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
@@ -459,6 +466,11 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
     p.eta = hp->eta;
     p.rs = make_rng_step(seed, step);
     p.prescaled = ctx->sh.per_node ? 1 : 0;
+    p.ecsgd = ecsgd ? 1 : 0;
+    if (ecsgd) {
+        p.wprime = reinterpret_cast<const float*>(ctx->base + ctx->ws.wplain);
+        p.eta = -hp->gamma;
+    }
 
     auto shape_of = [&](const Plan& pl, int mode) {
         LaunchShape s;
@@ -476,7 +488,7 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
         if (e == cudaSuccess) e = launch_finalize_scales(p, ctx->sh.code, stream);
     }
     if (e == cudaSuccess) {
-        const int kind = fused_kind(ctx);
+        const int kind = ecsgd ? 0 : fused_kind(ctx);
         if (kind == 2) {
             p.warps_per_group = ctx->tma.warps_per_group;
             p.nodes_per_block = ctx->tma.nodes_per_block;
@@ -518,6 +530,21 @@ ds_status ds_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, const d
                     uint64_t seed, uint64_t step, void* cuda_stream) {
     if (!ctx || !x || !delta || !g || !hp) return DS_ERR_NULL;
     return run_step(ctx, x, delta, g, nullptr, 0.0f, GRAD_GIVEN, hp, seed, step, cuda_stream);
+}
+
+ds_status ds_ecsgd_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, float gamma,
+                        uint64_t seed, uint64_t step, void* cuda_stream) {
+    if (!ctx || !x || !delta || !gp || !gp->a || !gp->c) return DS_ERR_NULL;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    const ds_hparams hp = {gamma, 0.0f};
+    return run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, gp->noise, &hp, seed, step, cuda_stream, 0, -1, true);
+}
+
+ds_status ds_ecsgd_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, float gamma,
+                          uint64_t seed, uint64_t step, void* cuda_stream) {
+    if (!ctx || !x || !delta || !g) return DS_ERR_NULL;
+    const ds_hparams hp = {gamma, 0.0f};
+    return run_step(ctx, x, delta, g, nullptr, 0.0f, GRAD_GIVEN, &hp, seed, step, cuda_stream, 0, -1, true);
 }
 
 ds_status ds_run(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const float* gammas,

@@ -14,6 +14,9 @@
 //                  nothing is re-read from global memory.
 //   MODE_COMPRESS  first half of the two-kernel path: writes x - gamma g into
 //                  x, delta', codes and scales; the mix kernel finishes.
+//                  With StepParams::ecsgd set it is the worker half of
+//                  centralized error-compensated SGD (Section 1): v = g + delta
+//                  is compressed, delta' and the codes are written, x is not.
 //   MODE_REDUCE    only the per-(node, tile) partial of the scale reduction
 //                  (used when one scale covers a whole node).
 //
@@ -179,10 +182,17 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
             const float4 a4 = ld4(p.a + row + e0);      // the gradient itself when it is given
             if constexpr (NOISE == GRAD_GIVEN) {
                 local_step4_given(x4, d4, a4, p.neg_gamma, &h[4 * r], &v[4 * r]);
+                if (MODE != MODE_FUSED && p.ecsgd) worker_step4_given(d4, a4, &v[4 * r]);
             } else {
                 const float4 c4 = ld4(p.c + row + e0);
                 const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + e0));
-                local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
+                if (MODE != MODE_FUSED && p.ecsgd) {
+                    worker_step4(x4, d4, a4, c4, z4, p.sigma, &v[4 * r]);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) h[4 * r + j] = 0.0f;
+                } else {
+                    local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
+                }
             }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -311,8 +321,10 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
                     }
                 }
                 st_partial(p.delta + row + e0, make_float4(dn[0], dn[1], dn[2], dn[3]), nv);
-                if constexpr (MODE == MODE_COMPRESS)
-                    st_partial(p.x + row + e0, make_float4(h[4 * r], h[4 * r + 1], h[4 * r + 2], h[4 * r + 3]), nv);
+                if constexpr (MODE == MODE_COMPRESS) {
+                    if (!p.ecsgd)
+                        st_partial(p.x + row + e0, make_float4(h[4 * r], h[4 * r + 1], h[4 * r + 2], h[4 * r + 3]), nv);
+                }
             }
             // gather the pieces of kLanesPerWord neighbouring lanes into one word
             uint32_t word = piece << ((4 * T::kBits * (lane % T::kLanesPerWord)) & 31);
@@ -324,7 +336,7 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
             }
         }
         if constexpr (T::kIdentity && MODE == MODE_COMPRESS) {
-            if (nv > 0)
+            if (nv > 0 && !p.ecsgd)
                 st_partial(p.x + row + e0, make_float4(h[4 * r], h[4 * r + 1], h[4 * r + 2], h[4 * r + 3]), nv);
         }
     }

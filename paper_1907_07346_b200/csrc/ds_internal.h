@@ -50,6 +50,8 @@ struct StepParams {
     int32_t warps_per_group;  // warps sharing one (node, tile)
     int32_t nodes_per_block;
     int32_t prescaled;        // 1: scale of node i is scales[i][0], computed by an earlier launch
+    int32_t ecsgd;            // 1 (compress / reduce modes only): centralized error-compensated SGD,
+                              // v = g + delta is compressed and x is left for the server's update
 };
 
 struct LaunchShape {
