@@ -99,7 +99,9 @@ typedef struct {
 typedef enum {
     DS_NOISE_NONE = 0,
     DS_NOISE_GAUSS = 1,         /* standard normal (Box-Muller) */
-    DS_NOISE_STUDENT_T3 = 2     /* Student t, 3 degrees of freedom, not re-normalised */
+    DS_NOISE_STUDENT_T3 = 2     /* Student t, 3 degrees of freedom, not re-normalised: consecutive
+                                   elements (2m, 2m+1) form a spherical bivariate t(3) pair
+                                   (each exactly t(3), uncorrelated, sharing one radius) */
 } ds_noise_kind;
 
 typedef struct {
@@ -274,11 +276,13 @@ ds_status ds_sync(ds_ctx *ctx, void *cuda_stream);
 /* Arithmetic self-test on the device the library runs on.  The noise kernels
  * replace two general routines by shortcuts that are exact only on the
  * arguments that can occur (a branch-free logarithm of j 2^-24 and a
- * one-correction square root of -2 ln u that starts from the hardware's
- * reciprocal-square-root estimate).  This runs both against the general forms
- * on ALL 2^24 possible arguments and ADDS the number of differing results to
- * counts[0] (logarithms) and counts[1] (square roots); counts is device memory,
- * two 64-bit integers, zeroed by the caller.  Both must stay 0. */
+ * one-correction square root, starting from the hardware's reciprocal-square-
+ * root estimate, of -2 ln u and of the squared Student-t(3) radius
+ * 3 (u^(-2/3) - 1)).  This runs them against the general forms on ALL 2^24
+ * possible arguments and ADDS the number of differing results to counts[0]
+ * (logarithms), counts[1] (roots of -2 ln u) and counts[2] (roots of the
+ * Student-t radii); counts is device memory, three 64-bit integers, zeroed by
+ * the caller.  All must stay 0. */
 ds_status ds_selftest_math(uint64_t *counts, void *cuda_stream);
 
 /* Failure-reporting self-test: enqueues a one-warp kernel that waits, with a

@@ -67,7 +67,7 @@ void oracle_philox4x32_10(const uint32_t ctr_in[4], const uint32_t key_in[2],
 }
 
 /*
- * Stream addressing (a convention of this build; the workload description
+ * Stream addressing (a convention of this library; the workload description
  * only says "keyed (seed, node, step, index)"):
  *   key     = (seed low 32 bits, seed high 32 bits)
  *   counter = (block, node, step low 32 bits, (step >> 32) << 8 | stream)
@@ -162,33 +162,67 @@ static void box_muller(uint32_t wa, uint32_t wb, float *z0, float *z1)
     *z1 = rho * s;
 }
 
+/* Radius of a Student-t(3) pair: sqrt(3 (u^(-2/3) - 1)) for u = j 2^-24,
+ * 1 <= j <= 2^24.  With theta uniform, (rho cos theta, rho sin theta) is then a
+ * spherical bivariate Student-t vector with 3 degrees of freedom (Bailey's
+ * polar method, Math. Comp. 62, 1994): both components are t(3) variates.
+ *   w = -(2/3) ln u >= 0;  k = nearest integer to w / ln 2;  r = w - k ln 2
+ *   (two-constant reduction, ln 2 = 0.693359375 - 2.1219444e-4);
+ *   expm1(r) = r + r^2 P(r), P of degree 5;
+ *   E = u^(-2/3) - 1 = 2^k expm1(r) + (2^k - 1)  (one fma: 2^k - 1 is exact);
+ *   rho = sqrt(3 E).
+ * The nearest integer is taken by adding and subtracting 1.5 * 2^23, which
+ * rounds to nearest-even in binary32 on every IEEE machine. */
+float oracle_t3_radius_u24(uint32_t j)
+{
+    float lg = oracle_log_u24(j);                       /* <= 0 */
+    float w = lg * -0x1.555556p-1f;
+    float t = fmaf(w, 0x1.715476p+0f, 12582912.0f);
+    float kf = t - 12582912.0f;
+    float r = fmaf(kf, -0.693359375f, w);
+    r = fmaf(kf, 0x1.bd0106p-13f, r);
+    float p = 0x1.9d1158p-13f;
+    p = fmaf(p, r, 0x1.6d7cc8p-10f);
+    p = fmaf(p, r, 0x1.111394p-7f);
+    p = fmaf(p, r, 0x1.5554a6p-5f);
+    p = fmaf(p, r, 0x1.555554p-3f);
+    p = fmaf(p, r, 0.5f);
+    float r2 = r * r;
+    float em = fmaf(r2, p, r);
+    float scale = ldexpf(1.0f, (int)kf);                /* 2^k, 0 <= k <= 16 */
+    float E = fmaf(scale, em, scale - 1.0f);
+    return sqrtf(3.0f * E);
+}
+
 enum { NOISE_NONE = 0, NOISE_GAUSS = 1, NOISE_STUDENT_T3 = 2 };
 
 /* Unit noise z for element k of a node (before the factor sigma).
- * GAUSS: block k/4 yields elements 4m..4m+3: words (0,1) -> 4m, 4m+1 and
- *        words (2,3) -> 4m+2, 4m+3.
- * STUDENT_T3: block k; (w0,w1) -> normals z0, z1; w2 -> a chi-square with two
- *        degrees of freedom e2 = -2 ln u; t = z0 / sqrt((z1^2 + e2)/3).
- *        (z1^2 + e2 is chi-square with three degrees of freedom.) */
+ * Block k/4 of the noise stream yields the elements 4m..4m+3: words (0,1) ->
+ * 4m, 4m+1 and words (2,3) -> 4m+2, 4m+3, each pair as
+ * (rho cos 2 pi u2, rho sin 2 pi u2) with u1 = ((wa >> 8) + 1) 2^-24,
+ * u2 = (wb >> 8) 2^-24 and
+ *   GAUSS:      rho = sqrt(-2 ln u1)              (Box-Muller: two independent normals)
+ *   STUDENT_T3: rho = sqrt(3 (u1^(-2/3) - 1))     (a spherical bivariate t(3) pair:
+ *               each element is exactly t(3)-distributed; the two elements of a
+ *               pair are uncorrelated but share their radius; pairs are independent). */
 float oracle_noise_elem(int kind, uint64_t seed, uint32_t node, uint64_t step,
                         int64_t k)
 {
     uint32_t w[4];
     float z0, z1;
-    if (kind == NOISE_GAUSS) {
+    if (kind == NOISE_GAUSS || kind == NOISE_STUDENT_T3) {
         philox_block(seed, node, step, STREAM_NOISE, (uint32_t)(k >> 2), w);
         int pair = (int)((k >> 1) & 1);
-        box_muller(w[2 * pair], w[2 * pair + 1], &z0, &z1);
+        if (kind == NOISE_GAUSS) {
+            box_muller(w[2 * pair], w[2 * pair + 1], &z0, &z1);
+        } else {
+            float rho = oracle_t3_radius_u24((w[2 * pair] >> 8) + 1u);
+            float c, s;
+            oracle_sincos_u24(w[2 * pair + 1] >> 8, &c, &s);
+            z0 = rho * c;
+            z1 = rho * s;
+        }
         return (k & 1) ? z1 : z0;
-    }
-    if (kind == NOISE_STUDENT_T3) {
-        philox_block(seed, node, step, STREAM_NOISE, (uint32_t)k, w);
-        box_muller(w[0], w[1], &z0, &z1);
-        float e2 = -2.0f * oracle_log_u24((w[2] >> 8) + 1u);
-        float q = fmaf(z1, z1, e2);
-        if (q == 0.0f) return 0.0f;
-        float d = sqrtf(q * 0x1.555556p-2f);
-        return z0 / d;
     }
     return 0.0f;
 }
@@ -549,6 +583,11 @@ int oracle_ecsgd_step(int32_t n, int64_t N, int64_t ld,
 void oracle_log_u24_array(uint32_t j0, int64_t count, float *out)
 {
     for (int64_t t = 0; t < count; ++t) out[t] = oracle_log_u24(j0 + (uint32_t)t);
+}
+
+void oracle_t3_radius_u24_array(uint32_t j0, int64_t count, float *out)
+{
+    for (int64_t t = 0; t < count; ++t) out[t] = oracle_t3_radius_u24(j0 + (uint32_t)t);
 }
 
 void oracle_sincos_u24_array(uint32_t k0, int64_t count, float *cos_out, float *sin_out)

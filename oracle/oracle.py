@@ -28,6 +28,8 @@ def lib():
         L.oracle_log_u24.restype = C.c_float
         L.oracle_log_u24_array.argtypes = [C.c_uint32, C.c_int64, _f32p]
         L.oracle_log_u24_array.restype = None
+        L.oracle_t3_radius_u24_array.argtypes = [C.c_uint32, C.c_int64, _f32p]
+        L.oracle_t3_radius_u24_array.restype = None
         L.oracle_sincos_u24_array.argtypes = [C.c_uint32, C.c_int64, _f32p, _f32p]
         L.oracle_sincos_u24_array.restype = None
         L.oracle_noise_row.argtypes = [C.c_int, C.c_uint64, C.c_uint32, C.c_uint64,
@@ -80,6 +82,13 @@ def philox(ctr, key):
 def log_u24_array(j0: int, count: int) -> np.ndarray:
     out = np.empty(count, dtype=np.float32)
     lib().oracle_log_u24_array(j0, count, _p(out, _f32p))
+    return out
+
+
+def t3_radius_u24_array(j0: int, count: int) -> np.ndarray:
+    """sqrt(3 ((j 2^-24)^(-2/3) - 1)) for j = j0 .. j0 + count - 1."""
+    out = np.empty(count, dtype=np.float32)
+    lib().oracle_t3_radius_u24_array(j0, count, _p(out, _f32p))
     return out
 
 

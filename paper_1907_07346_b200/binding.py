@@ -321,9 +321,10 @@ def ds_node_scales_noalloc(scales_out, x, delta, a, c, sigma: float, noise: int,
 
 
 def ds_selftest_math(stream=None):
-    """Run the arithmetic self-test; returns (differing logarithms, differing square roots)."""
+    """Run the arithmetic self-test; returns (differing logarithms, differing square
+    roots of -2 ln u, differing square roots of the Student-t radii)."""
     import torch
-    counts = torch.zeros(2, dtype=torch.int64, device="cuda")
+    counts = torch.zeros(3, dtype=torch.int64, device="cuda")
     s = torch.cuda.current_stream() if stream is None else stream
     _check(lib().ds_selftest_math(counts.data_ptr(), C.c_void_p(s.cuda_stream)), "ds_selftest_math")
     torch.cuda.synchronize()

@@ -9,6 +9,7 @@ codes have to match a plain IEEE evaluation bit for bit.
 from __future__ import annotations
 
 import os
+import re
 import subprocess
 import sys
 from concurrent.futures import ThreadPoolExecutor
@@ -19,27 +20,40 @@ OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdeepsqueeze.so")
 SOURCES = ["ds_api.cu", "ds_kernels_tma.cu", "ds_kernels_fused.cu", "ds_kernels_wide.cu", "ds_kernels_wide_tma.cu", "ds_kernels_compress.cu",
            "ds_kernels_misc.cu", "ds_noalloc.cu"]
-HEADERS = ["ds_device.cuh", "ds_internal.h", "ds_column_kernel.cuh", "ds_fused_tma_kernel.cuh", "ds_wide_fused_kernel.cuh", "ds_wide_tma_kernel.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-fmad=false", "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
 
 
-def _newest_input() -> float:
-    paths = [os.path.join(CSRC, f) for f in SOURCES + HEADERS]
-    paths.append(os.path.join(os.path.dirname(HERE), "include", "deepsqueeze.h"))
-    paths.append(os.path.abspath(__file__))
-    return max(os.path.getmtime(p) for p in paths)
+def _deps(path: str, seen: set | None = None) -> set:
+    """The file and every file it includes with #include "...", recursively."""
+    seen = set() if seen is None else seen
+    path = os.path.normpath(path)
+    if path in seen or not os.path.exists(path):
+        return seen
+    seen.add(path)
+    with open(path) as f:
+        for line in f:
+            m = re.match(r'\s*#\s*include\s+"([^"]+)"', line)
+            if m:
+                _deps(os.path.join(os.path.dirname(path), m.group(1)), seen)
+    return seen
+
+
+def _newest(paths) -> float:
+    return max(os.path.getmtime(p) for p in list(paths) + [os.path.abspath(__file__)])
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_input():
-        return LIB
     os.makedirs(OBJ, exist_ok=True)
     extra = ["-Xptxas", "-v"] if verbose else []
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ, src.replace(".cu", ".o"))
-        cmd = ["nvcc", *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
+        path = os.path.join(CSRC, src)
+        # an object is rebuilt when its source or anything it includes is newer
+        if not force and os.path.exists(obj) and os.path.getmtime(obj) >= _newest(_deps(path)):
+            return obj
+        cmd = ["nvcc", *NVCC_FLAGS, *extra, "-c", path, "-o", obj]
         res = subprocess.run(cmd, capture_output=True, text=True)
         if verbose or res.returncode != 0:
             sys.stderr.write(res.stdout + res.stderr)
@@ -49,8 +63,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
         objs = list(ex.map(compile_one, SOURCES))
-    subprocess.run(["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a",
-                    "-o", LIB, *objs], check=True)
+    if force or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
+        subprocess.run(["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a",
+                        "-o", LIB, *objs], check=True)
     return LIB
 
 

@@ -166,10 +166,10 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     float mn[kRndAhead ? E : 1];
     auto draw_noise = [&](int64_t c) {
         const uint32_t kbase = (uint32_t)(c * p.tile + seg0) + 4u * (uint32_t)lane;   // element of r = 0
-        if constexpr (NOISE == NOISE_GAUSS || (NOISE != NOISE_T3 && kRndAhead)) {
+        if constexpr (kNoiseAhead || kRndAhead) {
             // all Philox blocks of the tile (V for the noise, V for the rounding stream,
             // whichever are needed) advance together
-            constexpr int kGauss = (NOISE == NOISE_GAUSS) ? V : 0;
+            constexpr int kGauss = kNoiseAhead ? V : 0;
             constexpr int kRnd = kRndAhead ? V : 0;
             uint32_t stream[kGauss + kRnd], block[kGauss + kRnd];
             uint4 w[kGauss + kRnd];
@@ -182,42 +182,13 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
 #pragma unroll
             for (int r = 0; r < V; ++r) {
                 if constexpr (kGauss > 0) {
-                    const float4 z4 = box_muller_x2(w[r]);
+                    const float4 z4 = noise_of_block<NOISE>(w[r]);
                     zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
                 }
                 if constexpr (kRnd > 0) {
                     const uint4 u = w[kGauss + r];
                     mn[4 * r + 0] = __uint2float_rn(u.x >> 8); mn[4 * r + 1] = __uint2float_rn(u.y >> 8);
                     mn[4 * r + 2] = __uint2float_rn(u.z >> 8); mn[4 * r + 3] = __uint2float_rn(u.w >> 8);
-                }
-            }
-        } else if constexpr (NOISE == NOISE_T3 && kRndAhead) {
-            // per four elements: their four noise blocks and the rounding block together
-#pragma unroll
-            for (int r = 0; r < V; ++r) {
-                const uint32_t kr = kbase + 128u * (uint32_t)r;
-                const uint32_t stream[5] = {STREAM_NOISE, STREAM_NOISE, STREAM_NOISE, STREAM_NOISE, STREAM_ROUND};
-                const uint32_t block[5] = {kr, kr + 1u, kr + 2u, kr + 3u, kr >> 2};
-                uint4 w[5];
-                rng_blocks<5>(p.rs, (uint32_t)node, stream, block, w);
-                student_t3_pair(w[0], w[1], zn[4 * r + 0], zn[4 * r + 1]);
-                student_t3_pair(w[2], w[3], zn[4 * r + 2], zn[4 * r + 3]);
-                mn[4 * r + 0] = __uint2float_rn(w[4].x >> 8); mn[4 * r + 1] = __uint2float_rn(w[4].y >> 8);
-                mn[4 * r + 2] = __uint2float_rn(w[4].z >> 8); mn[4 * r + 3] = __uint2float_rn(w[4].w >> 8);
-            }
-        } else {
-            if constexpr (kRndAhead) {
-#pragma unroll
-                for (int r = 0; r < V; ++r) {
-                    const float4 rr = rnd24x4_unscaled(p.rs, (uint32_t)node, kbase + 128u * (uint32_t)r);
-                    mn[4 * r + 0] = rr.x; mn[4 * r + 1] = rr.y; mn[4 * r + 2] = rr.z; mn[4 * r + 3] = rr.w;
-                }
-            }
-            if constexpr (kNoiseAhead) {
-#pragma unroll
-                for (int r = 0; r < V; ++r) {
-                    const float4 z4 = noise4<NOISE>(p.rs, (uint32_t)node, kbase + 128u * (uint32_t)r);
-                    zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
                 }
             }
         }

@@ -175,10 +175,11 @@ __global__ void __launch_bounds__(32) ds_wait_selftest_kernel(int* error_flag) {
 // Self-test of the arithmetic shortcuts on every possible argument: the packed
 // branch-free logarithm against the scalar compare-and-halve form, and the
 // one-correction square root against sqrt.rn.f32, for all j = 1 .. 2^24.
-// counts[0] += mismatching logarithms, counts[1] += mismatching roots.
+// counts[0] += mismatching logarithms, counts[1] += mismatching roots,
+// counts[2] += mismatching roots of the Student-t(3) squared radii.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) ds_math_selftest_kernel(unsigned long long* counts) {
-    unsigned bad_log = 0, bad_sqrt = 0;
+    unsigned bad_log = 0, bad_sqrt = 0, bad_t3 = 0;
     for (uint32_t j = 1u + blockIdx.x * blockDim.x + threadIdx.x; j <= (1u << 24); j += gridDim.x * blockDim.x) {
         const uint32_t j2 = (j == (1u << 24)) ? 1u : j + 1u;
         const float2 lg = log_u24_x2(j, j2);
@@ -186,9 +187,12 @@ __global__ void __launch_bounds__(256) ds_math_selftest_kernel(unsigned long lon
         if (__float_as_uint(lg.y) != __float_as_uint(log_u24(j2))) ++bad_log;
         const float t = __fmul_rn(-2.0f, lg.x);
         if (__float_as_uint(sqrt_of_minus2log(t)) != __float_as_uint(__fsqrt_rn(t))) ++bad_sqrt;
+        const float2 q = t3_radius_sq_x2(j, j2);
+        if (__float_as_uint(sqrt_one_correction(q.x)) != __float_as_uint(__fsqrt_rn(q.x))) ++bad_t3;
     }
     if (bad_log) atomicAdd(&counts[0], (unsigned long long)bad_log);
     if (bad_sqrt) atomicAdd(&counts[1], (unsigned long long)bad_sqrt);
+    if (bad_t3) atomicAdd(&counts[2], (unsigned long long)bad_t3);
 }
 
 cudaError_t launch_math_selftest(unsigned long long* counts, cudaStream_t stream) {

@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
         return true;
     };
     // noise and rounding uniforms of item (col, b), Philox blocks in lockstep
-    constexpr bool kGaussAhead = (NOISE == NOISE_GAUSS);
+    constexpr bool kGaussAhead = (NOISE == NOISE_GAUSS || NOISE == NOISE_T3);
     constexpr bool kRndAhead = T::kLut;
     float zn[kGaussAhead ? E : 1];
     float mn[kRndAhead ? E : 1];
@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
 #pragma unroll
             for (int r = 0; r < V; ++r) {
                 if constexpr (kGa > 0) {
-                    const float4 z4 = box_muller_x2(w[r]);
+                    const float4 z4 = noise_of_block<NOISE>(w[r]);
                     zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
                 }
                 if constexpr (kRn > 0) {

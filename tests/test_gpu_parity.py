@@ -106,6 +106,19 @@ def test_noise_streams_bit_exact(env, noise):
     assert np.all(got[:, N:] == 0)
 
 
+@pytest.mark.parametrize("noise", [I.NOISE_GAUSS, I.NOISE_STUDENT_T3])
+def test_noise_streams_bit_exact_two_million_elements(env, noise):
+    """A long stretch of the stream (every exponent range of the radius occurs)."""
+    torch, orc, B = env
+    n, N = 2, 1 << 20
+    out = torch.zeros((n, N), dtype=torch.float32, device="cuda")
+    B.ds_noise(out, n, N, 0, noise, 31337, 12)
+    got = out.cpu().numpy()
+    for i in range(n):
+        ref = orc.noise_row(noise, 31337, i, 12, 0, N)
+        assert np.array_equal(got[i].view(np.uint32), ref.view(np.uint32))
+
+
 def test_rounding_stream_bit_exact(env):
     torch, orc, B = env
     n, N = 2, 1001
@@ -120,7 +133,7 @@ def test_arithmetic_shortcuts_exact_on_all_arguments(env):
     """The branch-free logarithm and the one-correction square root used by the
     noise kernels agree bit for bit with the general forms on all 2^24 arguments."""
     torch, orc, B = env
-    assert B.ds_selftest_math() == (0, 0)
+    assert B.ds_selftest_math() == (0, 0, 0)
 
 
 # ---------------------------------------------------------- single steps

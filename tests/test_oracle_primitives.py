@@ -137,7 +137,55 @@ def test_gauss_noise_is_standard_normal():
 def test_student_t3_noise_distribution():
     t = orc.noise_row(I.NOISE_STUDENT_T3, 77, 1, 4, 0, 1 << 19).astype(np.float64)
     assert stats.kstest(t[:200_000], "t", args=(3,)).pvalue > 1e-3
+    assert stats.kstest(t[1::2][:200_000], "t", args=(3,)).pvalue > 1e-3      # the sine halves alone
     assert abs(np.median(np.abs(t)) - stats.t.ppf(0.75, 3)) < 1e-2
+
+
+def test_student_t3_pairs_are_spherical_bivariate_t():
+    """(t_a, t_b) of a pair is a spherical bivariate t(3) vector: its squared
+    radius over 2 is F(2, 3)-distributed, its angle is uniform, and neither the
+    elements of a pair nor neighbouring pairs are correlated (checked on the
+    bounded transform tanh so that the heavy tails do not swamp the estimate)."""
+    t = orc.noise_row(I.NOISE_STUDENT_T3, 5, 0, 9, 0, 1 << 19).astype(np.float64).reshape(-1, 2)
+    rad2 = (t**2).sum(axis=1) / 2.0
+    assert stats.kstest(rad2[:200_000], "f", args=(2, 3)).pvalue > 1e-3
+    ang = np.arctan2(t[:, 1], t[:, 0])
+    assert stats.kstest(ang[:200_000], "uniform", args=(-np.pi, 2 * np.pi)).pvalue > 1e-3
+    b = np.tanh(t)
+    assert abs(np.corrcoef(b[:, 0], b[:, 1])[0, 1]) < 1e-2
+    assert abs(np.corrcoef(b[:-1, 1], b[1:, 0])[0, 1]) < 1e-2
+
+
+def test_student_t3_radius_accuracy_all_arguments():
+    """rho(j) = sqrt(3 ((j 2^-24)^(-2/3) - 1)) for every j = 1 .. 2^24 against
+    binary64: within 8 ulp, exact 0 at u = 1, largest value at j = 1."""
+    total = 1 << 24
+    blk = 1 << 22
+    worst = 0.0
+    for j0 in range(1, total + 1, blk):
+        got = orc.t3_radius_u24_array(j0, blk)
+        u = np.arange(j0, j0 + blk, dtype=np.float64) / total
+        ref = np.sqrt(3.0 * np.expm1(-(2.0 / 3.0) * np.log(u)))
+        ok = ref > 0
+        worst = max(worst, float(_ulp_err(got[ok], ref[ok]).max()))
+        assert np.all(got >= 0) and np.all(np.isfinite(got))
+    assert worst <= 8.0, worst
+    assert orc.t3_radius_u24_array(total, 1)[0] == 0.0
+    assert abs(orc.t3_radius_u24_array(1, 1)[0] - np.sqrt(3.0 * (2.0**16 - 1))) < 1e-3
+
+
+def test_student_t3_element_mapping():
+    """Element k takes words (0,1) or (2,3) of noise block k/4; the cosine
+    goes to the even element of the pair, the sine to the odd one."""
+    seed, node, step, N = 1234, 2, 7, 64
+    t = orc.noise_row(I.NOISE_STUDENT_T3, seed, node, step, 0, N)
+    for k in range(0, N, 2):
+        ctr = np.array([k >> 2, node, step, 0], dtype=np.uint32)
+        w = orc.philox(ctr, np.array([seed, 0], dtype=np.uint32))
+        pair = (k >> 1) & 1
+        rho = orc.t3_radius_u24_array((int(w[2 * pair]) >> 8) + 1, 1)[0]
+        c, s = orc.sincos_u24_array(int(w[2 * pair + 1]) >> 8, 1)
+        assert t[k] == np.float32(rho) * c[0] and t[k + 1] == np.float32(rho) * s[0]
 
 
 def test_noise_none_is_zero():
