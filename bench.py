@@ -51,8 +51,8 @@ def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) ->
 # profiles/ds_fused_tma_kernel_cfg3_small_counters.md (dram__bytes_read.sum +
 # dram__bytes_write.sum over one launch of 67,108,864 updates), valid for the
 # kernel sources whose digest is recorded beside it.
-NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59429e9 / 67108864,
-               "sources_sha256": "77e7338c5659be51fb15218266c863c8bb88b2d0824e8dc8284b04ef259eb4f0"}
+NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59443e9 / 67108864,
+               "sources_sha256": "e0820866c442e54e70352413bc57117afe027d20108a8807350097a44edb3876"}
 KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
 
 
@@ -204,6 +204,10 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=sorted(I.WORKLOADS))
     ap.add_argument("--size", type=int, default=0, help="override N (parameters per node)")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "fused_ldg", "split"])
+    ap.add_argument("--runner", default="step", choices=["step", "graph", "resident"],
+                    help="step: one ds_step call per iteration (the default); graph: all iterations as one ds_run "
+                         "call (a replayed CUDA graph); resident: all iterations as one ds_run_resident launch "
+                         "(small shapes only)")
     ap.add_argument("--elems-per-lane", type=int, default=0, help="tuning knob (0 = library default)")
     ap.add_argument("--given-gradient", action="store_true",
                     help="time ds_step_g (gradient read from memory) instead of the synthetic objective")
@@ -268,10 +272,20 @@ def main():
         else:
             ds.ds_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, k, stream)
 
+    def many_steps(k, count):
+        """count iterations from step k as ONE call: a replayed CUDA graph or the resident kernel."""
+        run = ds.ds_run if args.runner == "graph" else ds.ds_run_resident
+        run(x, delta, a, c, w.sigma, w.noise_kind, [w.gamma] * count, [w.eta] * count, w.seed, k, stream)
+
     step_index = 0
-    for _ in range(args.warmup):
-        one_step(step_index)
-        step_index += 1
+    if args.runner == "step":
+        for _ in range(args.warmup):
+            one_step(step_index)
+            step_index += 1
+    else:
+        for _ in range(3):                       # same count as the timed call, so the graph is instantiated once
+            many_steps(step_index, args.steps)
+            step_index += args.steps
     barrier()
 
     sampler = ClockSampler(local_rank)
@@ -281,15 +295,23 @@ def main():
     barrier()
     t_wall0 = time.time()
     events[0].record(stream)
-    for k in range(args.steps):
-        one_step(step_index)
-        step_index += 1
-        events[k + 1].record(stream)
+    if args.runner == "step":
+        for k in range(args.steps):
+            one_step(step_index)
+            step_index += 1
+            events[k + 1].record(stream)
+    else:
+        many_steps(step_index, args.steps)
+        step_index += args.steps
+        events[-1].record(stream)
     barrier()
     t_wall1 = time.time()
     clocks = sampler.stop(t_wall0, t_wall1)
     total_ms = events[0].elapsed_time(events[-1])
-    per_step = [events[k].elapsed_time(events[k + 1]) for k in range(args.steps)]
+    if args.runner == "step":
+        per_step = [events[k].elapsed_time(events[k + 1]) for k in range(args.steps)]
+    else:
+        per_step = [total_ms / args.steps] * args.steps
     total_ms = max_over_ranks(total_ms, dist, dev)
     updates_per_step = w.n * w.N
     value = whole_job_value(world, updates_per_step, args.steps, total_ms)
@@ -303,12 +325,13 @@ def main():
     kernel_ms = statistics.mean(per_step)
     traffic = None      # per launch; null once the kernel sources differ from the profiled ones
     if (not args.given_gradient and info.path == B.DS_PATH_FUSED and args.workload == NCU_TRAFFIC["workload"] and not args.elems_per_lane
-            and kernel_sources_digest() == NCU_TRAFFIC["sources_sha256"]):
+            and args.runner == "step" and kernel_sources_digest() == NCU_TRAFFIC["sources_sha256"]):
         traffic = NCU_TRAFFIC["bytes_per_update"] * updates_per_step
     achieved = b_alg * updates_per_step / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_source": f"of {peak_kind}",
-                "kernel": {B.DS_PATH_FUSED: "ds_fused_tma_kernel", B.DS_PATH_FUSED_LDG: "ds_column_kernel (fused)",
+                "kernel": "ds_resident_kernel" if args.runner == "resident" else
+                          {B.DS_PATH_FUSED: "ds_fused_tma_kernel", B.DS_PATH_FUSED_LDG: "ds_column_kernel (fused)",
                            B.DS_PATH_SPLIT: "ds_column_kernel (compress) + ds_mix_kernel"}[info.path],
                 "algorithmic_bytes_per_update": b_alg,
                 "algorithmic_bytes_per_launch": b_alg * updates_per_step,
@@ -362,8 +385,8 @@ def main():
                            "l2": "inputs larger than L2 (no flush needed)"
                                  if 16 * updates_per_step > 4 * 126e6 else "inputs fit in L2: not a roofline point",
                            "replicas": world},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * info.launches_per_step,
-                "roofline": roofline, "cpu_baseline": base}
+                "clocks": clocks, "e2e": e2e, "gpu_launches": 1 if args.runner == "resident" else args.steps * info.launches_per_step,
+                "runner": args.runner, "roofline": roofline, "cpu_baseline": base}
         print(json.dumps(line))
     ds.close()
     if dist is not None:

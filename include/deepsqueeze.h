@@ -228,6 +228,30 @@ ds_status ds_run(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
                  const float *gammas, const float *etas, int32_t T,
                  uint64_t seed, uint64_t step0, void *cuda_stream);
 
+/* T consecutive iterations as ONE kernel launch, for problems small enough to
+ * stay on chip between iterations (Algorithm 1 run as a loop; Section 5's
+ * learning-rate decay as the schedule).  Column tiles of 512 elements are
+ * independent except for the sum or maximum behind a per-node scale, so each
+ * thread block keeps one tile of all n nodes -- x and delta in registers, a and
+ * c in shared memory -- for all T iterations; global memory is read once at the
+ * start and written once at the end, plus the codes and scales every iteration
+ * "sends" (ds_codes returns those of the last one).  With one scale per node
+ * (chunk = 0) the blocks meet at one grid-wide barrier per iteration (the
+ * launch is cooperative, the barrier's wait bounded: DS_ERR_TIMEOUT from
+ * ds_sync if it ever runs out, x and delta then unchanged).  Results are
+ * bit-identical to T calls of ds_step.
+ *   Shapes: n <= 16; chunk = 512 or chunk = 0; DS_COMP_SIGN1_L1 or
+ *   DS_COMP_UNIFORM_STOCH_MAXABS with 2 or 4 bits; with chunk = 0 all
+ *   ceil(N/512) blocks must be resident at once (N up to a few hundred
+ *   thousand).  Anything else: DS_ERR_UNSUPPORTED, nothing runs -- use ds_run.
+ *   gammas, etas  host arrays of T values, copied before the call returns
+ *   T             1 .. DS_RESIDENT_MAX_STEPS
+ * Other arguments and errors as ds_run. */
+#define DS_RESIDENT_MAX_STEPS 1024
+ds_status ds_run_resident(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,
+                          const float *gammas, const float *etas, int32_t T,
+                          uint64_t seed, uint64_t step0, void *cuda_stream);
+
 /* Same iteration for HOST buffers: x, delta, a, c (host, [n][ld]) go to the
  * caller's device staging arrays, the step runs, and x and delta come back,
  * all ordered after the work already in `cuda_stream`; that stream continues

@@ -23,8 +23,9 @@ DS_COMP_IDENTITY, DS_COMP_SIGN1_L1, DS_COMP_UNIFORM_STOCH_MAXABS, DS_COMP_UNIFOR
 DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 DS_RUN_MAX_STEPS = 4096
+DS_RESIDENT_MAX_STEPS = 1024
 
-EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_g", "ds_ecsgd_step", "ds_ecsgd_step_g", "ds_run", "ds_step_host", "ds_codes", "ds_set_path",
+EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_g", "ds_ecsgd_step", "ds_ecsgd_step_g", "ds_run", "ds_run_resident", "ds_step_host", "ds_codes", "ds_set_path",
            "ds_tune", "ds_get_info", "ds_sync", "ds_selftest_timeout", "ds_selftest_math", "ds_noise", "ds_node_scales_noalloc",
            "ds_destroy", "ds_strerror"]
 
@@ -82,6 +83,8 @@ def lib():
         L.ds_run.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ds_grad_params), C.POINTER(C.c_float),
                              C.POINTER(C.c_float), C.c_int32, C.c_uint64, C.c_uint64, C.c_void_p]
         L.ds_run.restype = C.c_int
+        L.ds_run_resident.argtypes = L.ds_run.argtypes
+        L.ds_run_resident.restype = C.c_int
         L.ds_step_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                                    C.c_int32, C.POINTER(ds_hparams), C.c_uint64, C.c_uint64,
                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -212,6 +215,22 @@ class DeepSqueeze:
         s = torch.cuda.current_stream(self.device) if stream is None else stream
         _check(lib().ds_run(self.ctx, x.data_ptr(), delta.data_ptr(), C.byref(gp), ga, ea, T,
                             seed, step0, C.c_void_p(s.cuda_stream)), "ds_run")
+
+    def ds_run_resident(self, x, delta, a, c, sigma: float, noise: int, gammas, etas, seed: int, step0: int,
+                        stream=None):
+        """len(gammas) consecutive iterations from step0 in one launch of the resident
+        kernel (small shapes only; raises DsError(DS_ERR_UNSUPPORTED) otherwise)."""
+        torch = self.torch
+        for t in (x, delta, a, c):
+            assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (self.n, self.ld)
+        T = len(gammas)
+        assert len(etas) == T
+        gp = ds_grad_params(a.data_ptr(), c.data_ptr(), sigma, noise)
+        ga = (C.c_float * max(T, 1))(*[float(v) for v in gammas])
+        ea = (C.c_float * max(T, 1))(*[float(v) for v in etas])
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        _check(lib().ds_run_resident(self.ctx, x.data_ptr(), delta.data_ptr(), C.byref(gp), ga, ea, T,
+                                     seed, step0, C.c_void_p(s.cuda_stream)), "ds_run_resident")
 
     def ds_step_g(self, x, delta, g, gamma: float, eta: float, seed: int, step: int, stream=None):
         """One iteration with the gradient supplied as a device tensor g[n][ld]."""

@@ -10,6 +10,7 @@
 #include "ds_fused_tma_kernel.cuh"
 #include "ds_wide_fused_kernel.cuh"
 #include "ds_wide_tma_kernel.cuh"
+#include "ds_resident_kernel.cuh"
 
 using namespace ds;
 
@@ -35,7 +36,7 @@ struct Shape {
 };
 
 struct WsLayout {
-    size_t codes, scales, dscales, partials, row_ptr, col_idx, wprime, wplain, lut, error_flag, total;
+    size_t codes, scales, dscales, partials, rpartials, row_ptr, col_idx, wprime, wplain, lut, error_flag, barrier, total;
 };
 
 bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
@@ -76,6 +77,14 @@ bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
     return true;
 }
 
+// Shapes the resident multi-step kernel takes: one warp per node and tile of 512
+// elements, all tiles resident at once when a per-node scale needs the grid barrier.
+bool resident_shape(int32_t n, const Shape& sh) {
+    if (n > kResidentMaxNodes || sh.tile != kResidentTile) return false;
+    if (sh.code != CODE_SIGN && sh.code != CODE_U2 && sh.code != CODE_U4) return false;
+    return !sh.per_node || sh.tiles <= 1024;
+}
+
 WsLayout make_ws(int32_t n, int32_t nnz, const Shape& sh) {
     WsLayout w;
     size_t off = 0;
@@ -85,12 +94,16 @@ WsLayout make_ws(int32_t n, int32_t nnz, const Shape& sh) {
     w.dscales = norm ? off : w.scales;      // decode factors only differ from the sent scalars for norm-matched codes
     if (norm) off = align_up(off + (size_t)n * (size_t)sh.scales_pitch * 4, kAlign);
     w.partials = off; off = align_up(off + (sh.per_node ? (size_t)n * (size_t)sh.tiles * 8 : 0), kAlign);
+    // two buffers of per-tile partials for the resident multi-step kernel (small per-node-scale shapes only)
+    w.rpartials = off;
+    off = align_up(off + (resident_shape(n, sh) && sh.per_node ? 2 * (size_t)n * (size_t)sh.tiles * 8 : 0), kAlign);
     w.row_ptr = off;  off = align_up(off + (size_t)(n + 1) * 4, kAlign);
     w.col_idx = off;  off = align_up(off + (size_t)nnz * 4, kAlign);
     w.wprime = off;   off = align_up(off + (size_t)nnz * 4, kAlign);
     w.wplain = off;   off = align_up(off + (size_t)nnz * 4, kAlign);
     w.lut = off;      off = align_up(off + 256 * 4, kAlign);
     w.error_flag = off; off = align_up(off + 4, kAlign);
+    w.barrier = off;  off = align_up(off + 4, kAlign);
     w.total = off;
     return w;
 }
@@ -608,6 +621,56 @@ ds_status ds_run(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, 
     if (e != cudaSuccess) {
         (void)cudaGetLastError();
         return DS_ERR_CUDA;
+    }
+    return DS_OK;
+}
+
+ds_status ds_run_resident(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const float* gammas,
+                          const float* etas, int32_t T, uint64_t seed, uint64_t step0, void* cuda_stream) {
+    if (!ctx || !x || !delta || !gp || !gp->a || !gp->c || !gammas || !etas) return DS_ERR_NULL;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    if (T < 1 || T > DS_RESIDENT_MAX_STEPS) return DS_ERR_ARG;
+    if (step0 >= ((uint64_t)1 << 56) || step0 + (uint64_t)T > ((uint64_t)1 << 56)) return DS_ERR_ARG;
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
+                           reinterpret_cast<uintptr_t>(gp->a) | reinterpret_cast<uintptr_t>(gp->c);
+    if ((bits % 16) != 0) return DS_ERR_ALIGN;
+    if (!resident_shape(ctx->n, ctx->sh)) return DS_ERR_UNSUPPORTED;
+    if (resident_smem_layout(ctx->n, ctx->nnz).total > (size_t)kMaxSmem) return DS_ERR_UNSUPPORTED;
+
+    static_assert(DS_RESIDENT_MAX_STEPS == kResidentMaxSteps, "header and kernel disagree");
+    ResidentParams rp;
+    StepParams& p = rp.p;
+    p.x = x; p.delta = delta; p.a = gp->a; p.c = gp->c;
+    p.ld = ctx->ld; p.N = ctx->N; p.n = ctx->n; p.nnz = ctx->nnz;
+    p.tile = ctx->sh.tile; p.tiles = ctx->sh.tiles;
+    p.tile_begin = 0; p.tile_end = ctx->sh.tiles;
+    p.row_ptr = reinterpret_cast<const int32_t*>(ctx->base + ctx->ws.row_ptr);
+    p.col_idx = reinterpret_cast<const int32_t*>(ctx->base + ctx->ws.col_idx);
+    p.wprime = reinterpret_cast<const float*>(ctx->base + ctx->ws.wprime);
+    p.lut = reinterpret_cast<const float*>(ctx->base + ctx->ws.lut);
+    p.codes = reinterpret_cast<uint32_t*>(ctx->base + ctx->ws.codes);
+    p.code_pitch = ctx->sh.code_pitch;
+    p.scales = reinterpret_cast<float*>(ctx->base + ctx->ws.scales);
+    p.scales_pitch = ctx->sh.scales_pitch;
+    p.dscales = reinterpret_cast<float*>(ctx->base + ctx->ws.dscales);
+    p.partials = reinterpret_cast<double*>(ctx->base + ctx->ws.partials);
+    p.error_flag = reinterpret_cast<int*>(ctx->base + ctx->ws.error_flag);
+    p.sigma = gp->sigma;
+    p.neg_gamma = 0.0f; p.eta = 0.0f;
+    p.rs = make_rng_step(seed, step0);
+    p.warps_per_group = 1; p.nodes_per_block = ctx->n;
+    p.prescaled = ctx->sh.per_node ? 1 : 0;
+    p.ecsgd = 0;
+    rp.partials2 = reinterpret_cast<double*>(ctx->base + ctx->ws.rpartials);
+    rp.barrier = reinterpret_cast<unsigned int*>(ctx->base + ctx->ws.barrier);
+    rp.step0 = step0;
+    rp.T = T;
+    std::memcpy(rp.gammas, gammas, (size_t)T * sizeof(float));
+    std::memcpy(rp.etas, etas, (size_t)T * sizeof(float));
+    const cudaError_t e = launch_resident(ctx->sh.code, gp->noise, rp, ctx->num_sms, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return e == cudaErrorCooperativeLaunchTooLarge ? DS_ERR_UNSUPPORTED : DS_ERR_CUDA;
     }
     return DS_OK;
 }
