@@ -11,6 +11,7 @@
 #include "ds_wide_fused_kernel.cuh"
 #include "ds_wide_tma_kernel.cuh"
 #include "ds_resident_kernel.cuh"
+#include "ds_fused_tma_pair_kernel.cuh"
 
 using namespace ds;
 
@@ -169,6 +170,23 @@ Plan plan_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int force_e 
     return pl;
 }
 
+// Persistent TMA-staged kernel with two nodes per warp: 17..32 nodes, chunks of 256.
+Plan plan_tma_pair(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int force_e = 0) {
+    Plan pl;
+    pl.elems_per_lane = 8;
+    pl.warps_per_group = 1;
+    if (force_e != 0 && force_e != 8) return pl;
+    if (sh.tile != kPairTile || sh.per_node || n <= 16 || n > 32 || (n % 2) != 0 || num_sms < 1) return pl;
+    if (sh.code == CODE_ID32 || sh.code == CODE_N2 || sh.code == CODE_N4) return pl;
+    pl.nodes_per_block = n;
+    pl.block = dim3((unsigned)(n / 2 * 32));
+    pl.smem = tma_smem_layout(sh.code != CODE_SIGN, 16, n / 2, 1, kPairTile, n, nnz).total;
+    if (pl.smem > (size_t)kMaxSmem) return pl;
+    pl.grid = dim3((unsigned)std::min<int64_t>(sh.tiles, num_sms));
+    pl.ok = true;
+    return pl;
+}
+
 // Fused kernel that sweeps the nodes of a column in batches of nodes_per_block.
 Plan plan_wide(const Shape& sh, int32_t n, int32_t nnz, int force_e = 0) {
     Plan pl;
@@ -217,7 +235,7 @@ struct ds_ctx {
     WsLayout ws;
     unsigned char* base;
     int path_req;
-    Plan tma, wide_tma, fused, wide, compress, reduce;
+    Plan tma, tma_pair, wide_tma, fused, wide, compress, reduce;
     int num_sms;
     bool pipe_ready;                                  // streams / events of ds_step_host
     cudaStream_t pipe_stream[3];
@@ -332,6 +350,7 @@ ds_status ds_init(ds_ctx** out, const ds_graph* graph, const float* W, int32_t n
     }
     ctx->num_sms = sms;
     ctx->tma = plan_tma(sh, n, nnz, sms);
+    ctx->tma_pair = plan_tma_pair(sh, n, nnz, sms);
     ctx->wide_tma = plan_wide_tma(sh, n, nnz, sms);
     ctx->fused = plan_column(MODE_FUSED, sh, n, nnz);
     ctx->wide = plan_wide(sh, n, nnz);
@@ -376,11 +395,13 @@ void ds_destroy(ds_ctx* ctx) {
     delete ctx;
 }
 
-// 2: persistent TMA-staged fused kernel, 4: the same with the nodes in batches,
-// 1: fused kernel with direct loads, 3: the same in node batches, 0: two kernels
-static int fused_kind(const ds_ctx* ctx) {
+// 2: persistent TMA-staged fused kernel, 5: the same with two nodes per warp (synthetic
+// gradient only), 4: the same with the nodes in batches, 1: fused kernel with direct loads,
+// 3: the same in node batches, 0: two kernels
+static int fused_kind(const ds_ctx* ctx, bool grad_given = false) {
     if (ctx->path_req == DS_PATH_SPLIT) return 0;
     if (ctx->path_req != DS_PATH_FUSED_LDG) {
+        if (ctx->tma_pair.ok && !grad_given) return 5;
         if (ctx->tma.ok) return 2;
         if (ctx->wide_tma.ok) return 4;
     }
@@ -391,7 +412,7 @@ static int fused_kind(const ds_ctx* ctx) {
 ds_status ds_set_path(ds_ctx* ctx, int32_t path) {
     if (!ctx) return DS_ERR_NULL;
     if (path < DS_PATH_AUTO || path > DS_PATH_FUSED_LDG) return DS_ERR_ARG;
-    if (path == DS_PATH_FUSED && !ctx->fused.ok && !ctx->tma.ok && !ctx->wide.ok && !ctx->wide_tma.ok)
+    if (path == DS_PATH_FUSED && !ctx->fused.ok && !ctx->tma.ok && !ctx->tma_pair.ok && !ctx->wide.ok && !ctx->wide_tma.ok)
         return DS_ERR_UNSUPPORTED;
     if (path == DS_PATH_FUSED_LDG && !ctx->fused.ok && !ctx->wide.ok) return DS_ERR_UNSUPPORTED;
     ctx->path_req = path;
@@ -407,6 +428,7 @@ ds_status ds_tune(ds_ctx* ctx, int32_t elems_per_lane) {
     ctx->compress = compress;
     ctx->reduce = plan_column(MODE_REDUCE, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
     ctx->tma = plan_tma(ctx->sh, ctx->n, ctx->nnz, ctx->num_sms, elems_per_lane);
+    ctx->tma_pair = plan_tma_pair(ctx->sh, ctx->n, ctx->nnz, ctx->num_sms, elems_per_lane);
     ctx->wide_tma = plan_wide_tma(ctx->sh, ctx->n, ctx->nnz, ctx->num_sms, elems_per_lane);
     ctx->fused = plan_column(MODE_FUSED, ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
     ctx->wide = plan_wide(ctx->sh, ctx->n, ctx->nnz, elems_per_lane);
@@ -417,9 +439,9 @@ ds_status ds_get_info(const ds_ctx* ctx, ds_info* info) {
     if (!ctx || !info) return DS_ERR_NULL;
     const int kind = fused_kind(ctx);
     const bool fused = kind != 0;
-    const Plan& pl = (kind == 2) ? ctx->tma : (kind == 4) ? ctx->wide_tma : (kind == 1) ? ctx->fused
+    const Plan& pl = (kind == 2) ? ctx->tma : (kind == 5) ? ctx->tma_pair : (kind == 4) ? ctx->wide_tma : (kind == 1) ? ctx->fused
                    : (kind == 3) ? ctx->wide : ctx->compress;
-    info->path = (kind == 2 || kind == 4) ? DS_PATH_FUSED : (kind != 0) ? DS_PATH_FUSED_LDG : DS_PATH_SPLIT;
+    info->path = (kind == 2 || kind == 4 || kind == 5) ? DS_PATH_FUSED : (kind != 0) ? DS_PATH_FUSED_LDG : DS_PATH_SPLIT;
     info->node_batches = (kind == 3 || kind == 4) ? (ctx->n + pl.nodes_per_block - 1) / pl.nodes_per_block : 1;
     info->launches_per_step = (fused ? 1 : 2) + (ctx->sh.per_node ? 2 : 0);
     info->elems_per_lane = pl.elems_per_lane;
@@ -501,8 +523,12 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
         if (e == cudaSuccess) e = launch_finalize_scales(p, ctx->sh.code, stream);
     }
     if (e == cudaSuccess) {
-        const int kind = ecsgd ? 0 : fused_kind(ctx);
-        if (kind == 2) {
+        const int kind = ecsgd ? 0 : fused_kind(ctx, grad_kind == GRAD_GIVEN);
+        if (kind == 5) {
+            p.warps_per_group = 1;
+            p.nodes_per_block = ctx->n;
+            e = launch_fused_tma_pair(shape_of(ctx->tma_pair, MODE_FUSED), p, stream);
+        } else if (kind == 2) {
             p.warps_per_group = ctx->tma.warps_per_group;
             p.nodes_per_block = ctx->tma.nodes_per_block;
             e = launch_fused_tma(shape_of(ctx->tma, MODE_FUSED), p, stream);
