@@ -204,6 +204,9 @@ def main():
     ap.add_argument("--workload", default="cfg3", choices=sorted(I.WORKLOADS))
     ap.add_argument("--size", type=int, default=0, help="override N (parameters per node)")
     ap.add_argument("--path", default="auto", choices=["auto", "fused", "fused_ldg", "split"])
+    ap.add_argument("--algorithm", default="deepsqueeze", choices=["deepsqueeze", "ecsgd"],
+                    help="deepsqueeze: Algorithm 1 (the default, the headline metric); ecsgd: centralized "
+                         "error-compensated SGD of Section 1 (ds_ecsgd_step, two kernels per step)")
     ap.add_argument("--runner", default="step", choices=["step", "graph", "resident"],
                     help="step: one ds_step call per iteration (the default); graph: all iterations as one ds_run "
                          "call (a replayed CUDA graph); resident: all iterations as one ds_run_resident launch "
@@ -267,7 +270,9 @@ def main():
         torch.cuda.synchronize(dev)
 
     def one_step(k):
-        if args.given_gradient:       # a stands in for the caller's gradient array
+        if args.algorithm == "ecsgd":
+            ds.ds_ecsgd_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.seed, k, stream)
+        elif args.given_gradient:       # a stands in for the caller's gradient array
             ds.ds_step_g(x, delta, a, w.gamma, w.eta, w.seed, k, stream)
         else:
             ds.ds_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, k, stream)
@@ -325,12 +330,13 @@ def main():
     kernel_ms = statistics.mean(per_step)
     traffic = None      # per launch; null once the kernel sources differ from the profiled ones
     if (not args.given_gradient and info.path == B.DS_PATH_FUSED and args.workload == NCU_TRAFFIC["workload"] and not args.elems_per_lane
-            and args.runner == "step" and kernel_sources_digest() == NCU_TRAFFIC["sources_sha256"]):
+            and args.runner == "step" and args.algorithm == "deepsqueeze" and kernel_sources_digest() == NCU_TRAFFIC["sources_sha256"]):
         traffic = NCU_TRAFFIC["bytes_per_update"] * updates_per_step
     achieved = b_alg * updates_per_step / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_source": f"of {peak_kind}",
                 "kernel": "ds_resident_kernel" if args.runner == "resident" else
+                          "ds_column_kernel (compress, g + delta) + ds_mix_kernel (server update)" if args.algorithm == "ecsgd" else
                           {B.DS_PATH_FUSED: "ds_fused_tma_kernel", B.DS_PATH_FUSED_LDG: "ds_column_kernel (fused)",
                            B.DS_PATH_SPLIT: "ds_column_kernel (compress) + ds_mix_kernel"}[info.path],
                 "algorithmic_bytes_per_update": b_alg,
@@ -343,7 +349,7 @@ def main():
     # End to end through the host-buffer entry point: pinned host arrays in,
     # x and delta back out, every step.
     e2e = None
-    if not args.no_e2e and not args.given_gradient:
+    if not args.no_e2e and not args.given_gradient and args.algorithm == "deepsqueeze":
         hx = torch.zeros((w.n, ld), dtype=torch.float32).pin_memory()
         hd = torch.zeros((w.n, ld), dtype=torch.float32).pin_memory()
         ha = torch.from_numpy(a_h).pin_memory()
@@ -376,7 +382,8 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": w.describe() + (" [gradient given: ds_step_g]" if args.given_gradient else ""),
+                "config": {"workload": w.describe() + (" [gradient given: ds_step_g]" if args.given_gradient else "")
+                           + (" [centralized error-compensated SGD: ds_ecsgd_step]" if args.algorithm == "ecsgd" else ""),
                            "row_pitch": ld,
                            "path": {B.DS_PATH_FUSED: "fused (persistent, TMA-staged)",
                                     B.DS_PATH_FUSED_LDG: "fused (direct loads)", B.DS_PATH_SPLIT: "split"}[info.path],
@@ -385,7 +392,7 @@ def main():
                            "l2": "inputs larger than L2 (no flush needed)"
                                  if 16 * updates_per_step > 4 * 126e6 else "inputs fit in L2: not a roofline point",
                            "replicas": world},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": 1 if args.runner == "resident" else args.steps * info.launches_per_step,
+                "clocks": clocks, "e2e": e2e, "gpu_launches": 1 if args.runner == "resident" else args.steps * ((2 + (2 if w.chunk == 0 and w.comp_kind != I.COMP_IDENTITY else 0)) if args.algorithm == "ecsgd" else info.launches_per_step),
                 "runner": args.runner, "roofline": roofline, "cpu_baseline": base}
         print(json.dumps(line))
     ds.close()
