@@ -7,12 +7,14 @@
 // in registers, a_i and c_i in shared memory, and global memory is touched at
 // the start (load), at the end (store) and for what the nodes "send" (packed
 // codes and scales of every iteration).  Per iteration and warp:
-//   noise and rounding uniforms (Philox blocks in lockstep), local step,
-//   scale (per chunk: a warp reduction; per node: the tile's partial goes to
-//   global memory, ONE grid-wide barrier, every block then combines the
-//   partials of all tiles in the fixed order of the per-node finaliser),
-//   compression and residual, C[v] to shared memory, block barrier, local
-//   update from the neighbours' C[v], block barrier.
+//   local step with the noise drawn one iteration ahead; scale (per chunk: a
+//   warp reduction; per node: the tile's partial goes to global memory, the
+//   block ARRIVES at the one grid-wide barrier of the iteration, draws this
+//   iteration's rounding uniforms and the next iteration's noise -- neither
+//   depends on the scale -- with their Philox blocks in lockstep, and only then
+//   waits; every block combines the partials of all tiles in the fixed order of
+//   the per-node finaliser); compression and residual, C[v] to shared memory,
+//   block barrier, local update from the neighbours' C[v], block barrier.
 // The learning-rate schedule (gamma_t, eta_t) travels in the kernel parameters.
 //
 // The grid barrier is an arrival counter in the workspace; blocks are
@@ -117,7 +119,6 @@ __global__ void __launch_bounds__(MAXT, 1) ds_resident_kernel(const __grid_const
     }
     __syncthreads();
 
-    RngStep rs = p.rs;
     constexpr float kL = (float)((1u << (T::kBits & 15)) - 1u);
     constexpr float kHalfL = 0.5f * kL;
     constexpr bool kNoise = (NOISE == NOISE_GAUSS || NOISE == NOISE_T3);
@@ -125,39 +126,65 @@ __global__ void __launch_bounds__(MAXT, 1) ds_resident_kernel(const __grid_const
     const uint32_t kbase = (uint32_t)k0 + 4u * (uint32_t)lane;
     bool alive = true;
 
+    // Philox blocks of one node in lockstep, each with its own step and stream
+    // (words 2 and 3 of the counter): the rounding uniforms of iteration t are
+    // drawn together with the noise of iteration t + 1.
+    auto draw = [&](uint64_t step_round, uint64_t step_noise, bool want_noise, float (&zn)[kNoise ? E : 1],
+                    float (&mn)[kRnd ? E : 1]) {
+        if constexpr (kNoise || kRnd) {
+            constexpr int kNz = kNoise ? V : 0;
+            constexpr int kRn = kRnd ? V : 0;
+            uint32_t c0[kNz + kRn], c1[kNz + kRn], c2[kNz + kRn], c3[kNz + kRn];
+#pragma unroll
+            for (int r = 0; r < V; ++r) {
+                const uint32_t blk = (kbase + 128u * (uint32_t)r) >> 2;
+                if constexpr (kNz > 0) {
+                    c0[r] = blk; c1[r] = (uint32_t)node; c2[r] = (uint32_t)step_noise;
+                    c3[r] = (uint32_t)((step_noise >> 32) << 8) | STREAM_NOISE;
+                }
+                if constexpr (kRn > 0) {
+                    c0[kNz + r] = blk; c1[kNz + r] = (uint32_t)node; c2[kNz + r] = (uint32_t)step_round;
+                    c3[kNz + r] = (uint32_t)((step_round >> 32) << 8) | STREAM_ROUND;
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 10; ++q) {
+                const uint32_t ka = p.rs.k0[q], kb = p.rs.k1[q];
+#pragma unroll
+                for (int b = 0; b < kNz + kRn; ++b) {
+                    const uint64_t pa = (uint64_t)0xD2511F53u * c0[b];
+                    const uint64_t pb = (uint64_t)0xCD9E8D57u * c2[b];
+                    const uint32_t n0 = (uint32_t)(pb >> 32) ^ c1[b] ^ ka;
+                    const uint32_t n2 = (uint32_t)(pa >> 32) ^ c3[b] ^ kb;
+                    c1[b] = (uint32_t)pb;
+                    c3[b] = (uint32_t)pa;
+                    c0[b] = n0;
+                    c2[b] = n2;
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < V; ++r) {
+                if constexpr (kNz > 0) {
+                    if (want_noise) {
+                        const float4 z4 = noise_of_block<NOISE>(make_uint4(c0[r], c1[r], c2[r], c3[r]));
+                        zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
+                    }
+                }
+                if constexpr (kRn > 0) {
+                    mn[4 * r + 0] = __uint2float_rn(c0[kNz + r] >> 8); mn[4 * r + 1] = __uint2float_rn(c1[kNz + r] >> 8);
+                    mn[4 * r + 2] = __uint2float_rn(c2[kNz + r] >> 8); mn[4 * r + 3] = __uint2float_rn(c3[kNz + r] >> 8);
+                }
+            }
+        }
+    };
+
+    float zn[kNoise ? E : 1], mn[kRnd ? E : 1];
+    if constexpr (kNoise) draw(rp.step0, rp.step0, true, zn, mn);       // noise of the first iteration
+
     for (int t = 0; t < rp.T; ++t) {
         const float neg_gamma = -rp.gammas[t];
         const float eta = rp.etas[t];
         const uint64_t step = rp.step0 + (uint64_t)t;
-        rs.step_lo = (uint32_t)step;
-        rs.step_hi8 = (uint32_t)((step >> 32) << 8);
-
-        // ---- random numbers of the iteration ----
-        float zn[kNoise ? E : 1], mn[kRnd ? E : 1];
-        if constexpr (kNoise || kRnd) {
-            constexpr int kNz = kNoise ? V : 0;
-            constexpr int kRn = kRnd ? V : 0;
-            uint32_t stream[kNz + kRn], block[kNz + kRn];
-            uint4 w[kNz + kRn];
-#pragma unroll
-            for (int r = 0; r < V; ++r) {
-                if constexpr (kNz > 0) { stream[r] = STREAM_NOISE; block[r] = (kbase + 128u * (uint32_t)r) >> 2; }
-                if constexpr (kRn > 0) { stream[kNz + r] = STREAM_ROUND; block[kNz + r] = (kbase + 128u * (uint32_t)r) >> 2; }
-            }
-            rng_blocks<kNz + kRn>(rs, (uint32_t)node, stream, block, w);
-#pragma unroll
-            for (int r = 0; r < V; ++r) {
-                if constexpr (kNz > 0) {
-                    const float4 z4 = noise_of_block<NOISE>(w[r]);
-                    zn[4 * r + 0] = z4.x; zn[4 * r + 1] = z4.y; zn[4 * r + 2] = z4.z; zn[4 * r + 3] = z4.w;
-                }
-                if constexpr (kRn > 0) {
-                    const uint4 u = w[kNz + r];
-                    mn[4 * r + 0] = __uint2float_rn(u.x >> 8); mn[4 * r + 1] = __uint2float_rn(u.y >> 8);
-                    mn[4 * r + 2] = __uint2float_rn(u.z >> 8); mn[4 * r + 3] = __uint2float_rn(u.w >> 8);
-                }
-            }
-        }
 
         // ---- local step, scale partial ----
         float h[E], v[E];
@@ -184,15 +211,23 @@ __global__ void __launch_bounds__(MAXT, 1) ds_resident_kernel(const __grid_const
         if constexpr (T::kSign) part = warp_sum(sum);
         else part = (double)__uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
 
-        float s;
+        // one scale per node: publish the tile's partial and arrive at the grid barrier ...
+        double* mine = rp.partials2 + (size_t)(t & 1) * (size_t)p.n * (size_t)p.tiles;
         if (p.prescaled) {
-            // one scale per node: publish the tile's partial, meet every other block, combine all tiles
-            double* mine = rp.partials2 + (size_t)(t & 1) * (size_t)p.n * (size_t)p.tiles;
             if (lane == 0) mine[(size_t)node * (size_t)p.tiles + (size_t)col] = part;
             __syncthreads();
             if (threadIdx.x == 0) {
                 __threadfence();
                 atomicAdd(rp.barrier, 1u);
+            }
+        }
+        // ... draw what does not depend on the scale while the other blocks arrive:
+        // this iteration's rounding uniforms and the next iteration's noise
+        draw(step, step + 1u, t + 1 < rp.T, zn, mn);
+
+        float s;
+        if (p.prescaled) {
+            if (threadIdx.x == 0) {
                 const unsigned int target = (unsigned int)(t + 1) * gridDim.x;
                 bool ok = ld_acquire_gpu(rp.barrier) >= target;
                 if (!ok) {
@@ -208,6 +243,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_resident_kernel(const __grid_const
             __syncthreads();
             alive = flag_sm[0] != 0;
             if (!alive) break;
+            // every block combines the partials of all tiles in the order of the per-node finaliser
             const double* all = mine + (size_t)node * (size_t)p.tiles;
             double acc = 0.0;
             for (int64_t q = lane; q < p.tiles; q += 32) {
