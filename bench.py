@@ -326,6 +326,9 @@ def main():
     # Roofline of the dominant kernel.  On the fused path a step IS one launch
     # of the column kernel, so its average duration is the event time per step.
     b_alg = algorithmic_bytes_per_update(w, args.given_gradient)
+    # ds_ecsgd_step runs as one fused launch where the persistent kernel takes the shape with 16 elements per lane
+    ecsgd_fused = (args.algorithm == "ecsgd" and args.path == "auto" and info.path == B.DS_PATH_FUSED
+                   and info.elems_per_lane == 16 and info.block_threads <= 512 and info.node_batches == 1)
     peak, peak_kind = measured_peak()
     kernel_ms = statistics.mean(per_step)
     traffic = None      # per launch; null once the kernel sources differ from the profiled ones
@@ -336,6 +339,7 @@ def main():
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_source": f"of {peak_kind}",
                 "kernel": "ds_resident_kernel" if args.runner == "resident" else
+                          "ds_fused_tma_kernel (error-compensated SGD instantiation)" if ecsgd_fused else
                           "ds_column_kernel (compress, g + delta) + ds_mix_kernel (server update)" if args.algorithm == "ecsgd" else
                           {B.DS_PATH_FUSED: "ds_fused_tma_kernel", B.DS_PATH_FUSED_LDG: "ds_column_kernel (fused)",
                            B.DS_PATH_SPLIT: "ds_column_kernel (compress) + ds_mix_kernel"}[info.path],
@@ -392,7 +396,7 @@ def main():
                            "l2": "inputs larger than L2 (no flush needed)"
                                  if 16 * updates_per_step > 4 * 126e6 else "inputs fit in L2: not a roofline point",
                            "replicas": world},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": 1 if args.runner == "resident" else args.steps * ((2 + (2 if w.chunk == 0 and w.comp_kind != I.COMP_IDENTITY else 0)) if args.algorithm == "ecsgd" else info.launches_per_step),
+                "clocks": clocks, "e2e": e2e, "gpu_launches": 1 if args.runner == "resident" else args.steps * (((1 if ecsgd_fused else 2) + (2 if w.chunk == 0 and w.comp_kind != I.COMP_IDENTITY else 0)) if args.algorithm == "ecsgd" else info.launches_per_step),
                 "runner": args.runner, "roofline": roofline, "cpu_baseline": base}
         print(json.dumps(line))
     ds.close()

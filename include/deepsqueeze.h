@@ -200,10 +200,13 @@ ds_status ds_step_g(ds_ctx *ctx, float *x, float *delta, const float *g, const d
  * stay equal if they start equal).  Operation order per element:
  *     d = x - c; g = fma(a, d, sigma z); v = g + delta; compress; delta' = v - C;
  *     acc = 0; for j in N(i) ascending: acc = fma(W_ij, C_j, acc); x' = fma(-gamma, acc, x).
- * Always two kernels (the workers' compression, then the server's update, which
- * streams each worker's packed codes once); ds_set_path has no effect on it.
- * Traffic: 24 + b/8 + 4/chunk bytes per node-element plus the codes re-read by
- * the server ((deg+1) b/8, served by L2 where the codes fit).
+ * Where the persistent fused kernel takes the shape with 16 elements per lane
+ * and at most 512 threads (chunks of 512 elements or one scale per node, up to
+ * 16 nodes; chunks of 1024 up to 8 nodes; ...) the iteration is ONE launch of
+ * that kernel's error-compensated-SGD instantiation: 24 + b/8 + 4/chunk bytes
+ * per node-element.  Otherwise, and with ds_set_path(DS_PATH_SPLIT), two
+ * kernels: the workers' compression, then the server's update, which streams
+ * each worker's packed codes once and re-reads x (32 + (deg+2) b/8 bytes).
  * Arguments and errors as ds_step / ds_step_g; ds_codes returns what the
  * workers sent. */
 ds_status ds_ecsgd_step(ds_ctx *ctx, float *x, float *delta, const ds_grad_params *gp,

@@ -12,6 +12,7 @@
 #include "ds_wide_tma_kernel.cuh"
 #include "ds_resident_kernel.cuh"
 #include "ds_fused_tma_pair_kernel.cuh"
+#include "ds_fused_tma_ecsgd.h"
 
 using namespace ds;
 
@@ -523,8 +524,17 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
         if (e == cudaSuccess) e = launch_finalize_scales(p, ctx->sh.code, stream);
     }
     if (e == cudaSuccess) {
+        // centralized error-compensated SGD: the fused kernel where the shape allows
+        // (16 elements per lane, at most 512 threads), else two kernels
+        const bool ecsgd_fused = ecsgd && ctx->path_req != DS_PATH_SPLIT && ctx->path_req != DS_PATH_FUSED_LDG &&
+                                 ctx->tma.ok && ctx->tma.elems_per_lane == 16 && ctx->tma.block.x <= 512;
         const int kind = ecsgd ? 0 : fused_kind(ctx, grad_kind == GRAD_GIVEN);
-        if (kind == 5) {
+        if (ecsgd_fused) {
+            p.ecsgd = 0;          // the fused kernel is its own instantiation; the flag is for the two-kernel path
+            p.warps_per_group = ctx->tma.warps_per_group;
+            p.nodes_per_block = ctx->tma.nodes_per_block;
+            e = launch_fused_tma_ecsgd(shape_of(ctx->tma, MODE_FUSED), p, stream);
+        } else if (kind == 5) {
             p.warps_per_group = 1;
             p.nodes_per_block = ctx->n;
             e = launch_fused_tma_pair(shape_of(ctx->tma_pair, MODE_FUSED), p, stream);

@@ -96,7 +96,12 @@ __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-template <int CODE, int NOISE, int E, int MAXT>
+// EC = true: the iteration of centralized error-compensated SGD (Section 1)
+// on the same machinery: the compressed variable is v = g + delta, the value
+// kept for the update is x itself, and the launcher passes the weights W (not
+// W - I) and -gamma in the place of eta, so that the last phase computes
+// x' = fma(-gamma, sum_j W_ij C_j, x).
+template <int CODE, int NOISE, int E, int MAXT, bool EC = false>
 __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_constant__ StepParams p) {
     using T = CodeTraits<CODE>;
     constexpr int V = E / 4;
@@ -235,14 +240,17 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     const float4 d4 = *reinterpret_cast<const float4*>(slot_lane + 1 * SEG + 128 * r);
                     const float4 a4 = *reinterpret_cast<const float4*>(slot_lane + 2 * SEG + 128 * r);
                     if constexpr (NOISE == GRAD_GIVEN) {
-                        local_step4_given(x4, d4, a4, p.neg_gamma, &h[4 * r], &v[4 * r]);
+                        if constexpr (EC) worker_step4_given(d4, a4, &v[4 * r]);
+                        else local_step4_given(x4, d4, a4, p.neg_gamma, &h[4 * r], &v[4 * r]);
                     } else {
                         const float4 c4 = *reinterpret_cast<const float4*>(slot_lane + 3 * SEG + 128 * r);
                         float4 z4;
                         if constexpr (kNoiseAhead) z4 = make_float4(zn[4 * r + 0], zn[4 * r + 1], zn[4 * r + 2], zn[4 * r + 3]);
                         else z4 = noise4<NOISE>(p.rs, (uint32_t)node, (uint32_t)(k0 + seg0 + e0));
-                        local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
+                        if constexpr (EC) worker_step4(x4, d4, a4, c4, z4, p.sigma, &v[4 * r]);
+                        else local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, &h[4 * r], &v[4 * r]);
                     }
+                    if constexpr (EC) { h[4 * r + 0] = x4.x; h[4 * r + 1] = x4.y; h[4 * r + 2] = x4.z; h[4 * r + 3] = x4.w; }
     #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         if (!FULL && j >= nv) { h[4 * r + j] = 0.0f; v[4 * r + j] = 0.0f; }
@@ -442,6 +450,23 @@ cudaError_t launch_tma_one(const LaunchShape& sh, const StepParams& p, cudaStrea
         kern<<<sh.grid, sh.block, sh.smem, stream>>>(p);
     }
     return cudaGetLastError();
+}
+
+// Centralized error-compensated SGD: 16 elements per lane, blocks of up to 512 threads.
+template <int CODE>
+cudaError_t launch_tma_ecsgd_code(const LaunchShape& sh, const StepParams& p, cudaStream_t stream) {
+    if (sh.elems_per_lane != 16 || sh.block.x > 512) return cudaErrorInvalidValue;
+#define DS_TMA_EC_CASE(NZ) \
+    if (sh.noise == NZ) { \
+        auto kern = ds_fused_tma_kernel<CODE, NZ, 16, 512, true>; \
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sh.smem); \
+        if (e != cudaSuccess) return e; \
+        kern<<<sh.grid, sh.block, sh.smem, stream>>>(p); \
+        return cudaGetLastError(); \
+    }
+    DS_TMA_EC_CASE(NOISE_NONE) DS_TMA_EC_CASE(NOISE_GAUSS) DS_TMA_EC_CASE(NOISE_T3) DS_TMA_EC_CASE(GRAD_GIVEN)
+#undef DS_TMA_EC_CASE
+    return cudaErrorInvalidValue;
 }
 
 template <int CODE>

@@ -25,13 +25,14 @@ def env():
 
 
 def run_ecsgd(env, graph, N, kind, bits, chunk, noise, steps=1, seed=5, sigma=0.1, gamma=0.05,
-              tol=TOL_STEP, given=False, zero_start=False, equal_rows=False):
+              tol=TOL_STEP, given=False, zero_start=False, equal_rows=False, path=0):
     torch, orc, B = env
     ld = I.round_up(N, 4) + 8
     x, d, a, c = make_state(graph, N, ld, seed, zero_start=zero_start)
     if equal_rows:
         x[:, :N] = x[0, :N]
     ds = B.DeepSqueeze(graph, N, ld, kind, bits, chunk)
+    ds.ds_set_path(path)          # 0: the fused kernel where the shape allows; 2: always two kernels
     dev = [torch.from_numpy(t.copy()).cuda() for t in (x, d, a, c)]
     rng = np.random.default_rng(seed + 1)
     for t in range(steps):
@@ -64,18 +65,20 @@ COMPS = [(I.COMP_SIGN1_L1, 1, 128), (I.COMP_SIGN1_L1, 1, 0), (I.COMP_UNIFORM_STO
          (I.COMP_UNIFORM_STOCH_MAXABS, 8, 64), (I.COMP_UNIFORM_NEAREST_L2, 4, 96), (I.COMP_IDENTITY, 32, 0)]
 
 
+@pytest.mark.parametrize("path", [0, 2])
 @pytest.mark.parametrize("comp", COMPS)
 @pytest.mark.parametrize("noise", [I.NOISE_NONE, I.NOISE_GAUSS])
-def test_parameter_server_steps(env, comp, noise):
+def test_parameter_server_steps(env, comp, noise, path):
     """Complete graph with W = 1/n (the parameter server); several tiles and a ragged tail."""
     kind, bits, chunk = comp
-    run_ecsgd(env, I.complete(5), 512 * 5 + 40 + 3, kind, bits, chunk, noise, steps=3)
+    run_ecsgd(env, I.complete(5), 512 * 5 + 40 + 3, kind, bits, chunk, noise, steps=3, path=path)
 
 
+@pytest.mark.parametrize("path", [0, 2])
 @pytest.mark.parametrize("comp", [(I.COMP_SIGN1_L1, 1, 1024), (I.COMP_UNIFORM_STOCH_MAXABS, 4, 512)])
-def test_given_gradient(env, comp):
+def test_given_gradient(env, comp, path):
     kind, bits, chunk = comp
-    run_ecsgd(env, I.complete(4), 4096 + 17, kind, bits, chunk, I.NOISE_NONE, steps=2, given=True)
+    run_ecsgd(env, I.complete(4), 4096 + 17, kind, bits, chunk, I.NOISE_NONE, steps=2, given=True, path=path)
 
 
 def test_single_worker(env):
@@ -83,17 +86,20 @@ def test_single_worker(env):
     run_ecsgd(env, I.complete(1), 3000, I.COMP_UNIFORM_STOCH_MAXABS, 2, 128, I.NOISE_GAUSS, steps=3)
 
 
-def test_other_graphs_and_student_noise(env):
-    run_ecsgd(env, I.ring(7), 2048 + 40, I.COMP_UNIFORM_STOCH_MAXABS, 2, 256, I.NOISE_STUDENT_T3, steps=2)
-    run_ecsgd(env, I.torus(3, 4), 1500, I.COMP_SIGN1_L1, 1, 512, I.NOISE_GAUSS, steps=2)
+@pytest.mark.parametrize("path", [0, 2])
+def test_other_graphs_and_student_noise(env, path):
+    run_ecsgd(env, I.ring(7), 2048 + 40, I.COMP_UNIFORM_STOCH_MAXABS, 2, 256, I.NOISE_STUDENT_T3, steps=2, path=path)
+    run_ecsgd(env, I.torus(3, 4), 1500, I.COMP_SIGN1_L1, 1, 512, I.NOISE_GAUSS, steps=2, path=path)
+    run_ecsgd(env, I.ring(16), 512 * 400 + 40, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_GAUSS, steps=2, path=path)
 
 
 def test_twenty_free_running_steps_and_equal_rows(env):
     """Free-running from x = delta = 0; with the complete graph every worker's
     copy of the model stays the same row."""
-    gx = run_ecsgd(env, I.complete(8), 65536 // 8 + 24, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_GAUSS,
-                   steps=20, tol=TOL_RUN, zero_start=True)
-    assert np.array_equal(gx, np.broadcast_to(gx[0], gx.shape))
+    for path in (0, 2):
+        gx = run_ecsgd(env, I.complete(8), 65536 // 8 + 24, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_GAUSS,
+                       steps=20, tol=TOL_RUN, zero_start=True, path=path)
+        assert np.array_equal(gx, np.broadcast_to(gx[0], gx.shape))
 
 
 def test_deepsqueeze_step_unchanged_after_ecsgd(env):
