@@ -244,7 +244,9 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                         double* red = reinterpret_cast<double*>(smem + L.red_off) + red_parity * nwarps;
                         red_parity ^= 1;
                         if (lane == 0) red[warp] = part;
-                        __syncthreads();
+                        // only the G warps of this node meet (named barrier 1 + group): the other
+                        // groups of the block are not held back
+                        asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(32 * G) : "memory");
                         part = 0.0;
                         for (int w = 0; w < G; ++w) {
                             const double t = red[grp * G + w];
