@@ -16,9 +16,15 @@
 // packed codes and the scales still go to global memory: they are what the
 // node "sends".
 //
-// Every wait on an mbarrier is bounded.  A warp whose copy does not arrive
-// gives up, raises the step's error flag and drops out of the tile without
-// storing; the block leaves the tile loop together at the next barrier.
+// There is no block-wide barrier per tile: a warp announces "C[v] of my node
+// is in shared memory" on that node's mbarrier and waits only for the barriers
+// of its node's neighbours, so a block is not held to the pace of its slowest
+// warp.
+//
+// Every wait on an mbarrier is bounded.  A warp whose copy (or neighbour) does
+// not arrive gives up, raises the step's error flag and stops storing; from
+// then on it only keeps announcing its tiles, so that no other warp waits in
+// vain, and every warp that sees the flag does the same.
 #pragma once
 
 #include <type_traits>
@@ -28,7 +34,7 @@
 namespace ds {
 
 struct TmaSmemLayout {
-    uint32_t slots_off, cval_off, red_off, lut_off, rowptr_off, col_off, w_off, mbar_off, abort_off, total;
+    uint32_t slots_off, cval_off, red_off, lut_off, rowptr_off, col_off, w_off, mbar_off, nbar_off, abort_off, total;
     uint32_t seg_bytes;    // bytes of one array segment of one warp
 };
 
@@ -41,6 +47,7 @@ __host__ __device__ inline TmaSmemLayout tma_smem_layout(bool has_lut, int E, in
     L.cval_off = off;    off += 2u * (uint32_t)n * (uint32_t)tile * 4u;
     L.red_off = off;     off += (G > 1) ? (uint32_t)nwarps * 8u : 0u;
     L.mbar_off = off;    off += (uint32_t)nwarps * 8u;
+    L.nbar_off = off;    off += 2u * (uint32_t)n * 8u;      // "C[v] of node j is ready", one per buffer and node
     L.lut_off = off;     off += has_lut ? 256u * 4u : 0u;
     L.rowptr_off = off;  off += (uint32_t)(n + 1) * 4u;
     L.col_off = off;     off += (uint32_t)nnz * 4u;
@@ -59,6 +66,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -132,6 +142,9 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     for (int t = threadIdx.x; t < p.nnz; t += blockDim.x) { cj[t] = p.col_idx[t]; wp[t] = p.wprime[t]; }
     if (threadIdx.x < 2) abort_sm[threadIdx.x] = 0;
     if (lane == 0) mbar_init(bar, 1);
+    // one "ready" barrier per C[v] buffer and node, completed by the G warps of the node
+    const uint32_t nbar0 = smem_u32(smem + L.nbar_off);
+    for (int t = threadIdx.x; t < 2 * p.n; t += blockDim.x) mbar_init(nbar0 + 8u * (uint32_t)t, (uint32_t)G);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
@@ -201,10 +214,19 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     if (col < p.tile_end) draw_noise(col);      // (also when only the rounding stream is needed)
     uint32_t parity = 0;
     int buf = 0;
+    uint32_t iter = 0;          // tiles this block has worked on
+    bool drain = false;         // after an abort: keep announcing tiles so that no neighbour waits in vain, nothing else
     constexpr float kL = (float)((1u << (T::kBits & 15)) - 1u);
     constexpr float kHalfL = 0.5f * kL;
 
-    for (; col < p.tile_end; col += gridDim.x) {
+    for (; col < p.tile_end; col += gridDim.x, ++iter) {
+        if (drain) {
+            // (the block-wide barrier of the scale reduction of a multi-warp chunk is still kept)
+            if (G > 1 && !T::kIdentity && !p.prescaled) __syncthreads();
+            if (lane == 0) mbar_arrive(nbar0 + 8u * (uint32_t)(buf * p.n + node));
+            buf ^= 1;
+            continue;
+        }
         const int64_t k0 = col * p.tile;
         const int64_t remain = p.N - k0;
         const int m_len = (int)(remain < p.tile ? remain : p.tile);
@@ -389,8 +411,23 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 if constexpr (T::kNorm) p.dscales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = dscale;
             }
 
-            __syncthreads();       // C[v] of every node of this tile is in shared memory
-            if (abort_sm[buf]) return true;
+            // C[v] of this node is in shared memory: say so, then wait for the neighbours' only.
+            // (W is symmetric, so the nodes waited for are exactly the ones that read this node's
+            // C[v]: their arrival at the NEXT tile also tells that they are done reading this buffer
+            // before it is written again two tiles later.)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(nbar0 + 8u * (uint32_t)(buf * p.n + node));
+            {
+                const uint32_t nphase = (iter >> 1) & 1u;
+                bool ok = true;
+                for (int e = rp[node]; e < rp[node + 1]; ++e)
+                    ok = mbar_wait_bounded(nbar0 + 8u * (uint32_t)(buf * p.n + cj[e]), nphase) && ok;
+                if (!ok) {
+                    abort_sm[buf] = 1;
+                    if (lane == 0) *p.error_flag = 1;
+                }
+            }
+            if (abort_sm[0] | abort_sm[1]) return true;
 
             // ---- phase C: local update from the neighbours' C[v] ---------------
             float acc[E];
@@ -428,7 +465,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             return false;
         };
         const bool aborted = full ? tile_body(std::true_type{}) : tile_body(std::false_type{});
-        if (aborted) break;
+        if (aborted) drain = true;
         buf ^= 1;
     }
     // Leaving early (error path): let the copy that is still in flight land
