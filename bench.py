@@ -51,8 +51,8 @@ def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) ->
 # profiles/ds_fused_tma_kernel_cfg3_small_counters.md (dram__bytes_read.sum +
 # dram__bytes_write.sum over one launch of 67,108,864 updates), valid for the
 # kernel sources whose digest is recorded beside it.
-NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59370e9 / 67108864,
-               "sources_sha256": "a34086b52a21621f9fd584862757a06b80dbdbab7aefd19ee1bcf0c33b338421"}
+NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59466e9 / 67108864,
+               "sources_sha256": "320a09427ce41e0783c60676aa91cc18d84f8061d8266dc26f8a7f56f4153dd7"}
 KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
 
 
