@@ -24,7 +24,7 @@ def _rel(got, ref):
     return float((num / den).max())
 
 
-@pytest.mark.parametrize("name,N", [("cfg3", None), ("cfg2", None), ("cfg5", None), ("cfg4", 256 * 20000 + 40)])
+@pytest.mark.parametrize("name,N", [("cfg3", None), ("cfg2", None), ("cfg5", None), ("cfg4", None)])
 def test_full_size_windows(name, N):
     import torch
     from oracle import oracle as orc
