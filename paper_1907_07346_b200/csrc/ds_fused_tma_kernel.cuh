@@ -420,8 +420,10 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             {
                 const uint32_t nphase = (iter >> 1) & 1u;
                 bool ok = true;
-                for (int e = rp[node]; e < rp[node + 1]; ++e)
+                for (int e = rp[node]; e < rp[node + 1]; ++e) {
+                    if (G == 1 && cj[e] == node) continue;      // this warp wrote its own C[v]: __syncwarp() above orders it
                     ok = mbar_wait_bounded(nbar0 + 8u * (uint32_t)(buf * p.n + cj[e]), nphase) && ok;
+                }
                 if (!ok) {
                     abort_sm[buf] = 1;
                     if (lane == 0) *p.error_flag = 1;
