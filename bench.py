@@ -51,8 +51,8 @@ def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) ->
 # profiles/ds_fused_tma_kernel_cfg3_small_counters.md (dram__bytes_read.sum +
 # dram__bytes_write.sum over one launch of 67,108,864 updates), valid for the
 # kernel sources whose digest is recorded beside it.
-NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59429e9 / 67108864,
-               "sources_sha256": "605c90d0bafe2616ea011d5429462599c2c87bafabfd6f3ddcffa5f31e3b15e2"}
+NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59477e9 / 67108864,
+               "sources_sha256": "70a26dd3c0391f05e2eb5a296d21be63deab540aeaecb024c6077ee900865e51"}
 KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
 
 

@@ -102,6 +102,9 @@ __device__ __forceinline__ void norm_compress(const float* v, int valid_len, flo
     const bool fast = !dead && m >= 0x1p-60f && m <= 0x1p+60f;
     const float inv = fast ? __fdiv_rn(1.0f, m) : 0.0f;
     double sv2 = 0.0, sl2 = 0.0;
+    // level[q]^2 in binary64, stored behind the 16 levels of the table: a product of two binary32
+    // numbers is exact in binary64, so adding the stored square rounds exactly like the fused form
+    const double* lut_sq = reinterpret_cast<const double*>(lut + 32);
 #pragma unroll
     for (int t = 0; t < E; ++t) {
         const int k = 4 * (32 * (t >> 2) + lane) + (t & 3);
@@ -122,7 +125,7 @@ __device__ __forceinline__ void norm_compress(const float* v, int valid_len, flo
             // products of two binary32 numbers are exact in binary64, so the fused
             // form rounds exactly like "sum += product"
             sv2 = __fma_rn((double)v[t], (double)v[t], sv2);
-            sl2 = __fma_rn((double)cv[t], (double)cv[t], sl2);
+            sl2 = __dadd_rn(sl2, lut_sq[code]);
         }
     }
 #pragma unroll
@@ -425,6 +428,10 @@ __global__ void __launch_bounds__(1024, 1) ds_column_kernel(const __grid_constan
     if constexpr (T::kLut) {
         float* lut = reinterpret_cast<float*>(smem + L.lut_off);
         for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x) lut[t] = p.lut[t];
+        // norm-matched codes: squares of the levels in binary64 (exact), in the unused part of the table
+        if constexpr (T::kNorm)
+            for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x)
+                reinterpret_cast<double*>(lut + 32)[t] = (double)p.lut[t] * (double)p.lut[t];
     }
     if constexpr (MODE == MODE_FUSED) {
         int32_t* rp = reinterpret_cast<int32_t*>(smem + L.rowptr_off);

@@ -138,6 +138,10 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
 
     if constexpr (T::kLut)
         for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x) lut[t] = p.lut[t];
+        // norm-matched codes: squares of the levels in binary64 (exact), in the unused part of the table
+        if constexpr (T::kNorm)
+            for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x)
+                reinterpret_cast<double*>(lut + 32)[t] = (double)p.lut[t] * (double)p.lut[t];
     for (int t = threadIdx.x; t <= p.n; t += blockDim.x) rp[t] = p.row_ptr[t];
     for (int t = threadIdx.x; t < p.nnz; t += blockDim.x) { cj[t] = p.col_idx[t]; wp[t] = p.wprime[t]; }
     if (threadIdx.x < 2) abort_sm[threadIdx.x] = 0;
