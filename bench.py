@@ -47,10 +47,9 @@ def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) ->
     return (20.0 if given_gradient else 24.0) + bits / 8.0 + 4.0 / chunk
 
 
-# DRAM bytes per update of the dominant kernel from the ncu capture summarised in
-# profiles/ds_fused_tma_kernel_cfg3_small_counters.md (dram__bytes_read.sum +
-# dram__bytes_write.sum over one launch of 67,108,864 updates), valid for the
-# kernel sources whose digest is recorded beside it.
+# DRAM bytes per update of the dominant kernel from one ncu capture of a small case
+# (dram__bytes_read.sum + dram__bytes_write.sum over one launch of 67,108,864 updates,
+# scaled per update), valid for the kernel sources whose digest is recorded beside it.
 NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59477e9 / 67108864,
                "sources_sha256": "70a26dd3c0391f05e2eb5a296d21be63deab540aeaecb024c6077ee900865e51"}
 KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
@@ -173,17 +172,114 @@ def cpu_baseline(w: I.Workload, a: np.ndarray, c: np.ndarray, sample_cols: int, 
                       f"({w.n * cols} updates per step)"}, times
 
 
+def device_objective(torch, w: I.Workload, ld: int, dev):
+    """a, c drawn ON THE DEVICE from the workload's distributions (a ~ U[0.5, 2] or
+    10^U[-1, 1], c ~ N(0, 1)), padding columns zero.  For the secondary timing lines
+    only: the values do not come from inputs.objective(), which the headline run and
+    every parity test use."""
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(w.seed)
+    a = torch.zeros((w.n, ld), dtype=torch.float32, device=dev)
+    c = torch.zeros((w.n, ld), dtype=torch.float32, device=dev)
+    u = torch.rand((w.n, w.N), generator=gen, dtype=torch.float32, device=dev)
+    a[:, :w.N] = 0.5 + 1.5 * u if w.a_dist == "uniform" else torch.pow(10.0, 2.0 * u - 1.0)
+    del u
+    c[:, :w.N] = torch.randn((w.n, w.N), generator=gen, dtype=torch.float32, device=dev)
+    return a, c
+
+
+def timed_steps(torch, step_fn, first_step: int, steps: int, stream, dev, local_rank: int):
+    """Run step_fn(k) for k = first_step .. first_step+steps-1 with a CUDA event after
+    every call (on the launching stream) and the clock sampler running; returns
+    (per-step ms, total ms, clocks)."""
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    torch.cuda.synchronize(dev)
+    t0 = time.time()
+    events[0].record(stream)
+    for k in range(steps):
+        step_fn(first_step + k)
+        events[k + 1].record(stream)
+    torch.cuda.synchronize(dev)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    per_step = [events[k].elapsed_time(events[k + 1]) for k in range(steps)]
+    return per_step, events[0].elapsed_time(events[-1]), clocks
+
+
+KERNEL_OF = {"cfg1": "ds_column_kernel (reduce) + ds_finalize_scales_kernel + ds_fused_tma_kernel",
+             "cfg2": "ds_wide_tma_kernel", "cfg3": "ds_fused_tma_kernel", "cfg3_l2": "ds_fused_tma_kernel",
+             "cfg4": "ds_fused_tma_pair_kernel", "cfg5": "ds_wide_tma_kernel"}
+
+
+def other_workload_line(torch, B, name: str, steps: int, dev, local_rank: int, peak: float,
+                        algorithm: str = "deepsqueeze", shared=None):
+    """One secondary timing line: `steps` device-timed steps of another workload (or of
+    centralized error-compensated SGD on the headline shape) on its default path."""
+    w = I.WORKLOADS[name]
+    ld = I.row_pitch(w.N)
+    g = w.build_graph()
+    stream = torch.cuda.current_stream(dev)
+    if shared is not None:
+        a, c, x, delta = shared
+        x.zero_()
+        delta.zero_()
+        data = "a, c of the headline run (same shape and distributions)"
+    else:
+        a, c = device_objective(torch, w, ld, dev)
+        x = torch.zeros((w.n, ld), dtype=torch.float32, device=dev)
+        delta = torch.zeros_like(x)
+        data = "a, c drawn on the device from the workload's distributions (timing only)"
+    ds = B.DeepSqueeze(g, w.N, ld, w.comp_kind, w.bits, w.chunk, device=dev)
+    info = ds.ds_get_info()
+
+    def step_fn(k):
+        if algorithm == "ecsgd":
+            ds.ds_ecsgd_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.seed, k, stream)
+        else:
+            ds.ds_step(x, delta, a, c, w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, k, stream)
+
+    for k in range(5):
+        step_fn(k)
+    per_step, total_ms, clocks = timed_steps(torch, step_fn, 5, steps, stream, dev, local_rank)
+    ds.ds_sync(stream)
+    ok = bool(torch.isfinite(x).all()) and bool(torch.isfinite(delta).all())
+    b_alg = algorithmic_bytes_per_update(w)
+    ms = total_ms / steps
+    achieved = b_alg * w.n * w.N / (ms * 1e-3) / 1e9
+    desc = w.describe()
+    if w.noise_kind == I.NOISE_STUDENT_T3:
+        desc += " [t3 drawn as spherical pairs: elements 2m, 2m+1 share one radius]"
+    if algorithm == "ecsgd":
+        desc += " [centralized error-compensated SGD: ds_ecsgd_step]"
+    fused = info.path == B.DS_PATH_FUSED
+    kernel = (KERNEL_OF.get(name, "?") if fused else "not the TMA-staged path")
+    if algorithm == "ecsgd":
+        kernel = "ds_fused_tma_kernel (error-compensated SGD instantiation)"
+    line = {"workload": desc, "kernel": kernel, "steps": steps, "ms_per_step": ms,
+            "updates_per_s": w.n * w.N / (ms * 1e-3), "algorithmic_bytes_per_update": b_alg,
+            "achieved": achieved, "frac": achieved / peak,
+            "ms_first_last_10": [statistics.mean(per_step[:10]), statistics.mean(per_step[-10:])],
+            "block_threads": info.block_threads, "grid_blocks": info.grid_blocks, "node_batches": info.node_batches,
+            "clocks": clocks, "finite": ok, "data": data,
+            "l2": "inputs larger than L2" if 16 * w.n * w.N > 4 * 126e6 else "inputs fit in L2: not a roofline point"}
+    ds.close()
+    return line
+
+
 def run_reference(args, w: I.Workload):
     """The reference arm: the CPU checker on a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample = w.with_size(min(w.N, args.ref_cols))
+    sample = w.with_size(min(w.N, args.ref_cols) if args.ref_cols > 0 else w.N)
     a, c = I.objective(sample, I.row_pitch(sample.N))
     total = args.warmup + args.steps
     base, times = cpu_baseline(sample, a, c, sample.N, steps=total, full_N=w.N)
     timed = times[args.warmup:]
-    value = sample.n * min(sample.N, args.ref_cols) * len(timed) / sum(timed)
+    value = sample.n * sample.N * len(timed) / sum(timed)
     base["value"] = value
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * sum(timed) / len(timed),
@@ -219,8 +315,14 @@ def main():
     ap.add_argument("--cpu-steps", type=int, default=3, help="steps of the CPU-baseline sample")
     ap.add_argument("--cpu-cols", type=int, default=1 << 25,
                     help="columns per node of the CPU-baseline sample")
-    ap.add_argument("--ref-cols", type=int, default=1 << 21,
-                    help="columns per node of each step of --impl reference")
+    ap.add_argument("--ref-cols", type=int, default=0,
+                    help="columns per node of each step of --impl reference (0 = the whole workload)")
+    ap.add_argument("--sustained-steps", type=int, default=1000,
+                    help="steps of the sustained leg run after the headline region (0 = skip; 1 GPU only)")
+    ap.add_argument("--other-steps", type=int, default=50,
+                    help="timed steps of each secondary workload line (0 = skip; 1 GPU only)")
+    ap.add_argument("--cpu-single-cols", type=int, default=1 << 20,
+                    help="columns per node of the one-thread CPU-baseline sample (0 = skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -335,9 +437,15 @@ def main():
     if (not args.given_gradient and info.path == B.DS_PATH_FUSED and args.workload == NCU_TRAFFIC["workload"] and not args.elems_per_lane
             and args.runner == "step" and args.algorithm == "deepsqueeze" and kernel_sources_digest() == NCU_TRAFFIC["sources_sha256"]):
         traffic = NCU_TRAFFIC["bytes_per_update"] * updates_per_step
+    # `achieved` counts ALGORITHMIC bytes (what the step must move); `achieved_dram` counts the
+    # DRAM bytes the profiler saw for this kernel (less than algorithmic when the last written
+    # lines are still dirty in L2 at the end of the one captured launch).
     achieved = b_alg * updates_per_step / (kernel_ms * 1e-3) / 1e9
+    achieved_dram = None if traffic is None else traffic / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_source": f"of {peak_kind}",
+                "achieved_alg": achieved, "achieved_dram": achieved_dram,
+                "frac_dram": None if achieved_dram is None else achieved_dram / peak,
                 "kernel": "ds_resident_kernel" if args.runner == "resident" else
                           "ds_fused_tma_kernel (error-compensated SGD instantiation)" if ecsgd_fused else
                           "ds_column_kernel (compress, g + delta) + ds_mix_kernel (server update)" if args.algorithm == "ecsgd" else
@@ -349,6 +457,22 @@ def main():
                 "kernel_ms_median": statistics.median(per_step),
                 "kernel_ms_first_last_10": [statistics.mean(per_step[:10]), statistics.mean(per_step[-10:])],
                 "frac_of_nominal_8TBs": achieved / 8000.0}
+
+    # Sustained leg: the same kernel for long enough (>= 1.5 s) that the board's power
+    # management has settled; the headline region above is a short burst.
+    if world == 1 and args.sustained_steps > 0 and args.runner == "step":
+        sus_ms, sus_total, sus_clocks = timed_steps(torch, one_step, step_index, args.sustained_steps, stream, dev,
+                                                    local_rank)
+        step_index += args.sustained_steps
+        sus = sus_total / args.sustained_steps
+        sus_ach = b_alg * updates_per_step / (sus * 1e-3) / 1e9
+        roofline["sustained"] = {"steps": args.sustained_steps, "timed_region_s": sus_total * 1e-3, "ms_per_step": sus,
+                                 "updates_per_s": updates_per_step / (sus * 1e-3),
+                                 "achieved": sus_ach, "frac": sus_ach / peak,
+                                 "ms_first_last_10": [statistics.mean(sus_ms[:10]), statistics.mean(sus_ms[-10:])],
+                                 "sm_mhz": sus_clocks.get("sm_mhz"), "sm_max_mhz": sus_clocks.get("sm_max_mhz"),
+                                 "reasons": sus_clocks.get("reasons"), "samples": sus_clocks.get("samples")}
+        ds.ds_sync(stream)
 
     # End to end through the host-buffer entry point: pinned host arrays in,
     # x and delta back out, every step.
@@ -378,9 +502,34 @@ def main():
                               "pipelined: copy in / compute / copy out overlap)"}
         del hx, hd, ha, hc
 
+    # Secondary lines: the other workloads (and the headline shape's other modes), each on its
+    # default path, device-timed; context for the headline, not part of `value`.
+    others = None
+    if world == 1 and args.other_steps > 0 and args.workload == "cfg3" and not args.size and args.path == "auto" \
+            and args.algorithm == "deepsqueeze" and not args.given_gradient and not args.elems_per_lane:
+        others = []
+        shared = (a, c, x, delta)
+        others.append(other_workload_line(torch, B, "cfg3", args.other_steps, dev, local_rank, peak, "ecsgd", shared))
+        others.append(other_workload_line(torch, B, "cfg3_l2", args.other_steps, dev, local_rank, peak, shared=shared))
+        ds.close()
+        del shared, a, c, x, delta
+        torch.cuda.empty_cache()
+        for name in ("cfg2", "cfg4", "cfg5"):
+            others.append(other_workload_line(torch, B, name, args.other_steps, dev, local_rank, peak))
+            torch.cuda.empty_cache()
+
     base = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         base, _ = cpu_baseline(w, a_h, c_h, args.cpu_cols, steps=args.cpu_steps)
+        if args.cpu_single_cols > 0:
+            from oracle import oracle as orc
+            threads = orc.num_threads()
+            orc.set_num_threads(1)
+            try:
+                single, _ = cpu_baseline(w, a_h, c_h, args.cpu_single_cols, steps=1)
+            finally:
+                orc.set_num_threads(threads)
+            base["single_thread"] = {"value": single["value"], "unit": UNIT, "cores": 1, "sample": single["sample"]}
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -397,7 +546,7 @@ def main():
                                  if 16 * updates_per_step > 4 * 126e6 else "inputs fit in L2: not a roofline point",
                            "replicas": world},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": 1 if args.runner == "resident" else args.steps * (((1 if ecsgd_fused else 2) + (2 if w.chunk == 0 and w.comp_kind != I.COMP_IDENTITY else 0)) if args.algorithm == "ecsgd" else info.launches_per_step),
-                "runner": args.runner, "roofline": roofline, "cpu_baseline": base}
+                "runner": args.runner, "roofline": roofline, "cpu_baseline": base, "other_workloads": others}
         print(json.dumps(line))
     ds.close()
     if dist is not None:

@@ -343,8 +343,9 @@ ds_status ds_noise(float *out, int32_t n, int64_t N, int64_t ld_out, int32_t whi
  * device [n][ld] arrays as for ds_step and are only read.
  *
  * The reduction's scratch is a fixed array inside the library
- * (DS_NOALLOC_MAX_PARTIALS binary64 partials plus a 1 KiB table, 544 KiB, held on
- * every GPU that loads the library until the process exits).  Consequences:
+ * (DS_NOALLOC_MAX_PARTIALS binary64 partials plus a 1 KiB table, 513 KiB, held on
+ * every GPU on which this entry point has been called, until the process exits).
+ * Consequences:
  *   - sizes with n * ceil(N / 512) > DS_NOALLOC_MAX_PARTIALS are rejected with
  *     DS_ERR_WORKSPACE;
  *   - all calls on one GPU share the array, so two calls whose kernels can
@@ -352,8 +353,10 @@ ds_status ds_noise(float *out, int32_t n, int64_t N, int64_t ld_out, int32_t whi
  *   - the array keeps the previous call's contents, which is harmless: each call
  *     overwrites every partial it later reads;
  *   - the first call on each device looks up the array's device address (with
- *     that device current); make that first call before starting any stream
- *     capture.
+ *     that device current), and that lookup is also the moment the driver gives
+ *     the array its storage on that GPU: make the first call at start-up, before
+ *     the GPU has been filled (it returns DS_ERR_CUDA if the 513 KiB cannot be
+ *     had) and before starting any stream capture.
  * The call allocates nothing: no cudaMalloc, cudaFree or allocating library
  * routine.  It only enqueues two kernels on cuda_stream. */
 #define DS_NOALLOC_MAX_PARTIALS 65536

@@ -622,3 +622,14 @@ int oracle_num_threads(void)
 #endif
     return t;
 }
+
+/* Host threads the (node, chunk) work items are spread over from now on
+ * (the benchmark times the oracle on one thread and on all cores). */
+void oracle_set_num_threads(int t)
+{
+#ifdef _OPENMP
+    if (t >= 1) omp_set_num_threads(t);
+#else
+    (void)t;
+#endif
+}

@@ -63,6 +63,8 @@ def lib():
         L.oracle_ecsgd_step.restype = C.c_int
         L.oracle_num_threads.argtypes = []
         L.oracle_num_threads.restype = C.c_int
+        L.oracle_set_num_threads.argtypes = [C.c_int]
+        L.oracle_set_num_threads.restype = None
         _lib = L
     return _lib
 
@@ -210,3 +212,8 @@ def ecsgd_step(graph, comp_kind: int, bits: int, chunk: int, x: np.ndarray, delt
 
 def num_threads() -> int:
     return int(lib().oracle_num_threads())
+
+
+def set_num_threads(t: int) -> None:
+    """Spread the (node, chunk) work items over t host threads from now on."""
+    lib().oracle_set_num_threads(int(t))

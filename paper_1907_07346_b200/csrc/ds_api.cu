@@ -762,6 +762,7 @@ ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const floa
     cudaError_t e = cudaEventRecord(ev_start, stream);
     for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(ctx->pipe_stream[i], ev_start, 0);
     const int64_t per = (tiles + slabs - 1) / slabs;
+    ds_status failed = DS_OK;
     for (int sidx = 0; sidx < slabs && e == cudaSuccess; ++sidx) {
         const int64_t t0 = sidx * per, t1 = std::min<int64_t>(tiles, t0 + per);
         if (t0 >= t1) break;
@@ -776,8 +777,8 @@ ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const floa
         if (e == cudaSuccess) e = cudaEventRecord(ctx->pipe_event[2 * sidx], s_in);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(s_run, ctx->pipe_event[2 * sidx], 0);
         if (e != cudaSuccess) break;
-        const ds_status st = run_step(ctx, dev_x, dev_delta, dev_a, dev_c, sigma, noise, hp, seed, step, s_run, t0, t1);
-        if (st != DS_OK) return st;
+        failed = run_step(ctx, dev_x, dev_delta, dev_a, dev_c, sigma, noise, hp, seed, step, s_run, t0, t1);
+        if (failed != DS_OK) break;
         e = cudaEventRecord(ctx->pipe_event[2 * sidx + 1], s_run);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, ctx->pipe_event[2 * sidx + 1], 0);
         if (e == cudaSuccess)
@@ -787,10 +788,32 @@ ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const floa
             e = cudaMemcpy2DAsync(delta_host + c0, pitch, dev_delta + c0, pitch, (size_t)c_out * sizeof(float),
                                   (size_t)ctx->n, cudaMemcpyDeviceToHost, s_out);
     }
+    if (failed != DS_OK || e != cudaSuccess) {
+        // Error path: copies and kernels already enqueued on the internal streams may still be
+        // touching the caller's buffers.  Whatever was enqueued is joined into the caller's
+        // stream before the error is returned, so that the caller's next work on that stream
+        // (or its synchronisation) is ordered after all of it.
+        (void)cudaGetLastError();
+        cudaEvent_t ev_in = ctx->pipe_event[0], ev_run = ctx->pipe_event[1];
+        bool joined = cudaEventRecord(ev_in, s_in) == cudaSuccess && cudaStreamWaitEvent(s_out, ev_in, 0) == cudaSuccess &&
+                      cudaEventRecord(ev_run, s_run) == cudaSuccess && cudaStreamWaitEvent(s_out, ev_run, 0) == cudaSuccess &&
+                      cudaEventRecord(ev_done, s_out) == cudaSuccess && cudaStreamWaitEvent(stream, ev_done, 0) == cudaSuccess;
+        if (!joined) {
+            (void)cudaGetLastError();
+            for (int i = 0; i < 3; ++i) (void)cudaStreamSynchronize(ctx->pipe_stream[i]);   // last resort: wait here
+            (void)cudaGetLastError();
+        }
+        return failed != DS_OK ? failed : DS_ERR_CUDA;
+    }
     // the caller's stream continues when the last slab is back (which implies every earlier stage)
-    if (e == cudaSuccess) e = cudaEventRecord(ev_done, s_out);
+    e = cudaEventRecord(ev_done, s_out);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ev_done, 0);
-    if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        for (int i = 0; i < 3; ++i) (void)cudaStreamSynchronize(ctx->pipe_stream[i]);
+        (void)cudaGetLastError();
+        return DS_ERR_CUDA;
+    }
     return DS_OK;
 }
 

@@ -86,13 +86,18 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 }
 // Bounded wait: false if the phase did not complete within `limit_ns` of
 // wall-clock time (and at most 2^22 polls).  In steady state the first poll
-// succeeds and the timer is never read.
+// succeeds and the timer is never read.  `gave_up` (optional): two flags in
+// shared memory that a warp of the block raises when ITS wait ran out; the
+// slow path polls them, so that once one warp has given up the others stop
+// waiting at once instead of each spending its own full time limit.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
-                                                  uint64_t limit_ns = 2000000000ull) {
+                                                  uint64_t limit_ns = 2000000000ull,
+                                                  const volatile int* gave_up = nullptr) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (uint32_t tries = 0; tries < (1u << 22); ++tries) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (gave_up != nullptr && (gave_up[0] | gave_up[1]) != 0) return false;
         if (global_timer_ns() - t0 > limit_ns) return false;
     }
     return false;
@@ -426,7 +431,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 bool ok = true;
                 for (int e = rp[node]; e < rp[node + 1]; ++e) {
                     if (G == 1 && cj[e] == node) continue;      // this warp wrote its own C[v]: __syncwarp() above orders it
-                    ok = mbar_wait_bounded(nbar0 + 8u * (uint32_t)(buf * p.n + cj[e]), nphase) && ok;
+                    ok = mbar_wait_bounded(nbar0 + 8u * (uint32_t)(buf * p.n + cj[e]), nphase, 2000000000ull, abort_sm) && ok;
                 }
                 if (!ok) {
                     abort_sm[buf] = 1;

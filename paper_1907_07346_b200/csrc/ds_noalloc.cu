@@ -17,8 +17,10 @@ namespace {
 
 // Layout of the static scratch (binary64 slots): the first kTableSlots hold a
 // zero table that the reduction kernel copies but never uses, the rest hold the
-// per-(node, tile) partials.  544 KiB in total, resident on every GPU that
-// loads the library until the process exits.
+// per-(node, tile) partials.  (128 + 65,536) * 8 B = 513 KiB in total.  The array is
+// part of this module's image: with lazy module loading the driver gives it
+// storage on a GPU when the module is first used there, i.e. at the first
+// cudaGetSymbolAddress below, and keeps it until the process exits.
 constexpr int64_t kTableSlots = 128;                 // 1 KiB
 constexpr int64_t kMaxPartials = DS_NOALLOC_MAX_PARTIALS;
 constexpr int kMaxDevices = 64;

@@ -24,16 +24,31 @@ def _rel(got, ref):
     return float((num / den).max())
 
 
-@pytest.mark.parametrize("name,N", [("cfg3", None), ("cfg2", None), ("cfg5", None), ("cfg4", None)])
-def test_full_size_windows(name, N):
+def _device_outputs(torch, ds):
+    """Views (no copy) of the packed codes and scales the last step left in the workspace."""
+    cptr, cpitch, sptr, spitch = ds.ds_codes()
+    base = ds.workspace.data_ptr()
+    codes = ds.workspace[cptr - base: cptr - base + ds.n * cpitch * 4].view(torch.int32).view(ds.n, cpitch)
+    scales = ds.workspace[sptr - base: sptr - base + ds.n * spitch * 4].view(torch.int32).view(ds.n, spitch)
+    return codes, scales
+
+
+@pytest.mark.parametrize("name", ["cfg3", "cfg2", "cfg5", "cfg4"])
+def test_full_size_windows_and_paths(name):
+    """Two free-running steps at the workload's full size on the default path (the kernel the
+    benchmark times).  (1) 64 seeded random chunk columns plus windows at the start, in the
+    middle and at the ragged end of the rows against the oracle: codes bit-exact, floats
+    bit-exact for max-abs scales, within 1e-5 for l1 scales.  (2) The WHOLE arrays -- x, delta,
+    packed codes, scales -- against the two-kernel path run from the same state, compared
+    bit for bit on the device: the two paths share the canonical operation order, the scale
+    of a chunk is summed in the same lane order, so any difference is a defect of one of them."""
     import torch
     from oracle import oracle as orc
     from paper_1907_07346_b200 import binding as B
     from paper_1907_07346_b200 import build as libbuild
+    from test_gpu_parity import assert_state_matches
     libbuild.build()
     w = I.WORKLOADS[name]
-    if N is not None:
-        w = w.with_size(N)
     N = w.N
     g = w.build_graph()
     ld = I.row_pitch(N)
@@ -48,35 +63,56 @@ def test_full_size_windows(name, N):
                 arr[i, :N] = rng.standard_normal(N, dtype=np.float32) * np.float32(
                     {"x": 0.3, "d": 0.05, "c": 1.0}[kind])
         host.append(arr)
-    ds = B.DeepSqueeze(g, N, ld, w.comp_kind, w.bits, w.chunk)
-    dev = [torch.from_numpy(t).cuda() for t in host]
     steps = 2
     chunk = w.chunk
     M = (N + chunk - 1) // chunk
     bits = 1 if w.comp_kind == I.COMP_SIGN1_L1 else w.bits
     windows = [(0, 4 * chunk), ((M // 2) * chunk, 3 * chunk), ((M - 3) * chunk, N - (M - 3) * chunk)]
+    pick = np.random.default_rng(w.seed + 7).choice(M - 1, size=64, replace=False)
+    windows += [(int(m) * chunk, chunk) for m in sorted(pick)]
     # oracle state per window, advanced alongside the GPU
     wstate = []
     for k0, cols in windows:
         sl = slice(k0, k0 + cols)
         wstate.append([np.ascontiguousarray(h[:, sl]) for h in host])
-    for t in range(steps):
-        ds.ds_step(dev[0], dev[1], dev[2], dev[3], w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, t)
-        ds.ds_sync()
-        codes, scales = ds.codes_to_host()
-        gx, gd = dev[0].cpu().numpy(), dev[1].cpu().numpy()
-        assert np.isfinite(gx).all() and np.isfinite(gd).all()
-        assert np.all(gx[:, N:] == 0) and np.all(gd[:, N:] == 0)          # padding untouched
-        for (k0, cols), st in zip(windows, wstate):
-            cw, sw, _, _ = orc.step(g, w.comp_kind, w.bits, chunk, st[0], st[1], st[2], st[3], cols,
-                                    w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, t, k_first=k0)
-            w0 = k0 * bits // 32
-            assert np.array_equal(codes[:, w0:w0 + cw.shape[1]], cw), (name, t, k0)
-            m0 = k0 // chunk
-            assert _rel(scales[:, m0:m0 + sw.shape[1]], sw) <= TOL
-            assert _rel(gx[:, k0:k0 + cols], st[0]) <= TOL, (name, t, k0)
-            assert _rel(gd[:, k0:k0 + cols], st[1]) <= TOL, (name, t, k0)
-    ds.close()
+
+    results = {}
+    for path in (B.DS_PATH_AUTO, B.DS_PATH_SPLIT):
+        ds = B.DeepSqueeze(g, N, ld, w.comp_kind, w.bits, w.chunk)
+        ds.ds_set_path(path)
+        if path == B.DS_PATH_AUTO:
+            assert ds.ds_get_info().path == B.DS_PATH_FUSED and ds.ds_get_info().grid_blocks == 148
+        dev = [torch.from_numpy(t).cuda() for t in host]
+        clean = [None] * len(windows)
+        for t in range(steps):
+            ds.ds_step(dev[0], dev[1], dev[2], dev[3], w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, t)
+            ds.ds_sync()
+            if path != B.DS_PATH_AUTO:
+                continue
+            assert bool(torch.isfinite(dev[0]).all()) and bool(torch.isfinite(dev[1]).all())
+            assert bool((dev[0][:, N:] == 0).all()) and bool((dev[1][:, N:] == 0).all())     # padding untouched
+            codes_d, scales_d = _device_outputs(torch, ds)
+            for wi, ((k0, cols), st) in enumerate(zip(windows, wstate)):
+                cw, sw, _, _ = orc.step(g, w.comp_kind, w.bits, chunk, st[0], st[1], st[2], st[3], cols,
+                                        w.sigma, w.noise_kind, w.gamma, w.eta, w.seed, t, k_first=k0)
+                w0 = k0 * bits // 32
+                got_codes = codes_d[:, w0:w0 + cw.shape[1]].cpu().numpy().view(np.uint32)
+                assert np.array_equal(got_codes, cw), (name, t, k0)
+                m0 = k0 // chunk
+                got_scales = scales_d[:, m0:m0 + sw.shape[1]].cpu().numpy().view(np.float32)
+                gx = dev[0][:, k0:k0 + cols].cpu().numpy()
+                gd = dev[1][:, k0:k0 + cols].cpu().numpy()
+                clean[wi] = assert_state_matches(w.comp_kind, cols, chunk, (gx, gd, got_scales),
+                                                 (st[0], st[1], sw), TOL, f"{name} step {t} column {k0}", clean[wi])
+        codes_d, scales_d = _device_outputs(torch, ds)
+        words = (N * bits + 31) // 32
+        results[path] = (dev[0], dev[1], codes_d[:, :words].clone(), scales_d[:, :M].clone())
+        del dev
+        ds.close()
+    for u, v, what in zip(results[B.DS_PATH_AUTO], results[B.DS_PATH_SPLIT], ("x", "delta", "codes", "scales")):
+        if u.dtype == torch.float32:
+            u, v = u.view(torch.int32), v.view(torch.int32)
+        assert torch.equal(u, v), f"{name}: {what} of the fused and the two-kernel path differ"
 
 
 def test_host_buffer_entry_point_pipelined():

@@ -54,8 +54,44 @@ def make_state(graph, N, ld, seed, a_dist="uniform", zero_start=False):
     return x, d, a, c
 
 
+def assert_state_matches(kind, N, chunk, got, ref, tol, where="", clean=None):
+    """got, ref = (x, delta, scales) of the GPU and of the oracle, [n][>= N] / [n][M].
+
+    A max-abs scale is an exact maximum and the identity compressor has no scale, so there
+    every float of x, delta and the scales must agree BIT FOR BIT.  An l1 scale (and the
+    norms of the norm-matched codec) is a binary64 sum rounded once to binary32, whose last
+    bit may depend on the order of the sum: scales within `tol`, x and delta within `tol`
+    per node row, and bit for bit in every chunk column whose scales have come out
+    identical so far (`clean`, one flag per chunk column, carried from step to step of a
+    free-running comparison; returned updated)."""
+    gx, gd, gs = got
+    rx, rd, rs = ref
+    if kind in (I.COMP_UNIFORM_STOCH_MAXABS, I.COMP_IDENTITY):
+        if kind != I.COMP_IDENTITY:
+            assert np.array_equal(gs.view(np.uint32), rs.view(np.uint32)), f"scales differ {where}"
+        assert np.array_equal(gx[:, :N].view(np.uint32), rx[:, :N].view(np.uint32)), f"x differs {where}"
+        assert np.array_equal(gd[:, :N].view(np.uint32), rd[:, :N].view(np.uint32)), f"delta differs {where}"
+        return clean
+    assert row_rel_err(gs, rs) <= tol, f"scales {where}"
+    ex, ed = row_rel_err(gx[:, :N], rx[:, :N]), row_rel_err(gd[:, :N], rd[:, :N])
+    assert ex <= tol and ed <= tol, (where, ex, ed)
+    same = np.all(gs.view(np.uint32) == rs.view(np.uint32), axis=0)          # per chunk column
+    clean = same if clean is None else (clean & same)
+    ch = chunk if chunk > 0 else N
+    mask = np.repeat(clean, ch)[:N]
+    assert np.array_equal(gx[:, :N].view(np.uint32)[:, mask], rx[:, :N].view(np.uint32)[:, mask]), f"x {where}"
+    assert np.array_equal(gd[:, :N].view(np.uint32)[:, mask], rd[:, :N].view(np.uint32)[:, mask]), f"delta {where}"
+    # an order-dependent last bit is rare: nearly all columns must still be identical
+    assert clean.size < 100 or clean.mean() >= 0.99, (where, clean.mean())
+    return clean
+
+
 def run_case(env, graph, N, kind, bits, chunk, noise, path, steps=1, pad=None, seed=3,
-             sigma=0.1, gamma=0.05, eta=0.5, zero_start=False, tol=TOL_STEP, a_dist="uniform"):
+             sigma=0.1, gamma=0.05, eta=0.5, zero_start=False, tol=TOL_STEP, a_dist="uniform",
+             allow_ldg=False):
+    """`path` is the path asked for; DS_PATH_FUSED must resolve to a TMA-staged kernel unless
+    allow_ldg says that this shape is known to have none (then the direct-load fused kernel
+    runs and the case is a second test of it)."""
     torch, orc, B = env
     ld = I.round_up(N, 4) + (0 if pad is None else pad)
     x, d, a, c = make_state(graph, N, ld, seed, a_dist, zero_start)
@@ -70,9 +106,12 @@ def run_case(env, graph, N, kind, bits, chunk, noise, path, steps=1, pad=None, s
     except B.DsError:
         ds.close()
         pytest.skip("shape not available on the fused path")
-    assert ds.ds_get_info().path == path or (path == B.DS_PATH_FUSED and ds.ds_get_info().path == B.DS_PATH_FUSED_LDG)
+    resolved = ds.ds_get_info().path
+    if resolved != path:
+        assert allow_ldg and path == B.DS_PATH_FUSED and resolved == B.DS_PATH_FUSED_LDG, \
+            f"asked for path {path}, the library resolved it to {resolved}"
     dev = [torch.from_numpy(t.copy()).cuda() for t in (x, d, a, c)]
-    worst = 0.0
+    clean = None
     for t in range(steps):
         codes_ref, scales_ref, _, _ = orc.step(graph, kind, bits, chunk, x, d, a, c, N, sigma, noise,
                                                gamma, eta, 99 + seed, t)
@@ -81,14 +120,10 @@ def run_case(env, graph, N, kind, bits, chunk, noise, path, steps=1, pad=None, s
         gx, gd = dev[0].cpu().numpy(), dev[1].cpu().numpy()
         codes, scales = ds.codes_to_host()
         assert np.array_equal(codes, codes_ref), f"codes differ at step {t}"
-        if kind != I.COMP_IDENTITY:
-            assert row_rel_err(scales, scales_ref) <= tol
-        ex, ed = row_rel_err(gx[:, :N], x[:, :N]), row_rel_err(gd[:, :N], d[:, :N])
-        worst = max(worst, ex, ed)
-        assert ex <= tol and ed <= tol, (t, ex, ed)
+        clean = assert_state_matches(kind, N, chunk, (gx, gd, scales), (x, d, scales_ref), tol,
+                                     f"at step {t}", clean)
         assert np.array_equal(gx[:, N:], x[:, N:]) and np.array_equal(gd[:, N:], d[:, N:])
     ds.close()
-    return worst
 
 
 # ------------------------------------------------------------ raw streams
@@ -309,6 +344,7 @@ def test_given_gradient_steps(env, path, case):
         pytest.skip("shape not available on this path")
     dx, dd = torch.from_numpy(x.copy()).cuda(), torch.from_numpy(d.copy()).cuda()
     zeros = np.zeros_like(x)
+    clean = None
     for t in range(3):
         grad = np.zeros_like(x)
         grad[:, :N] = rng.standard_normal((g.n, N)).astype(np.float32)
@@ -319,9 +355,9 @@ def test_given_gradient_steps(env, path, case):
         ds.ds_sync()
         codes, scales = ds.codes_to_host()
         assert np.array_equal(codes, codes_ref)
-        assert row_rel_err(scales, scales_ref) <= TOL_STEP
         gx, gd = dx.cpu().numpy(), dd.cpu().numpy()
-        assert row_rel_err(gx[:, :N], x[:, :N]) <= TOL_STEP and row_rel_err(gd[:, :N], d[:, :N]) <= TOL_STEP
+        clean = assert_state_matches(kind, N, chunk, (gx, gd, scales), (x, d, scales_ref), TOL_STEP,
+                                     f"at step {t}", clean)
         assert np.array_equal(gx[:, N:], x[:, N:]) and np.array_equal(gd[:, N:], d[:, N:])
     ds.close()
 

@@ -1,5 +1,6 @@
 """The allocation-free entry point ds_node_scales_noalloc against the regular
-per-node-scale path (ds_step with chunk = 0, scales read back via ds_codes).
+per-node-scale path (ds_step with chunk = 0, scales read back via ds_codes)
+and against the CPU oracle's per-node scales (independent code).
 
 Collected last on purpose: if it fails, a run that stops at the first failure
 has already run every other test.  The entry point keeps its scratch in a
@@ -13,7 +14,7 @@ from paper_1907_07346_b200 import inputs as I
 
 pytestmark = pytest.mark.gpu
 
-TOL = 1e-5      # the tolerance of the parity tests; the two paths run the same kernels
+TOL = 1e-5      # the tolerance of the parity tests (l1 scales; max-abs scales are compared bit for bit)
 
 
 def _reference_scales(torch, B, g, N, ld, kind, bits, arrays, sigma, noise, gamma, seed, step):
@@ -27,26 +28,51 @@ def _reference_scales(torch, B, g, N, ld, kind, bits, arrays, sigma, noise, gamm
     return scales[:, 0]
 
 
+def _oracle_scales(g, N, kind, bits, host, sigma, noise, gamma, seed, step):
+    """Per-node scales of the CPU oracle: one step with chunk = 0 on copies."""
+    from oracle import oracle as orc
+    cp = [h.copy() for h in host]
+    _, scales, _, _ = orc.step(g, kind, bits, 0, cp[0], cp[1], cp[2], cp[3], N, sigma, noise, gamma, 0.5,
+                               seed, step)
+    return scales[:, 0]
+
+
+def _assert_scales(kind, got, want, what):
+    if kind == I.COMP_UNIFORM_STOCH_MAXABS:          # an exact maximum: no tolerance
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), (what, got, want)
+    else:                                            # a binary64 sum rounded once to binary32
+        assert np.abs(got - want).max() <= TOL * np.abs(want).max(), (what, got, want)
+
+
+# (graph, noise, pitch beyond N rounded up to 4, sizes of the two calls)
+CASES = [(I.ring(8), I.NOISE_GAUSS, 0, [(512 * 9 + 37, 11), (512 * 2 + 5, 12)]),
+         # more than one batch of nodes per grid row, a padded pitch, the other noise kinds
+         (I.ring(12), I.NOISE_STUDENT_T3, 8, [(512 * 3 + 100, 21), (512 * 7 + 1, 22)]),
+         (I.ring(3), I.NOISE_NONE, 4, [(515, 31), (40, 32)])]
+
+
 @pytest.mark.parametrize("kind,bits", [(I.COMP_SIGN1_L1, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 4)])
-def test_noalloc_scales_match_regular_path_twice(kind, bits):
+@pytest.mark.parametrize("case", CASES, ids=["ring8-gauss", "ring12-t3-padded", "ring3-nonoise"])
+def test_noalloc_scales_match_regular_path_and_oracle_twice(kind, bits, case):
     import torch
     from paper_1907_07346_b200 import binding as B
     from paper_1907_07346_b200 import build as libbuild
     libbuild.build()
-    g = I.ring(8)
-    sigma, noise, gamma = 0.1, I.NOISE_GAUSS, 0.05
+    g, noise, pad, calls = case
+    sigma, gamma = 0.1, 0.05
     out = torch.full((g.n,), -1.0, dtype=torch.float32, device="cuda")
-    # two calls in a row: a larger problem first, then a smaller one with other data
-    for call, (N, seed) in enumerate([(512 * 9 + 37, 11), (512 * 2 + 5, 12)]):
-        ld = I.round_up(N, 4)
+    # two calls in a row on different sizes and data: nothing of the first may leak into the second
+    for call, (N, seed) in enumerate(calls):
+        ld = I.round_up(N, 4) + pad
         rng = np.random.default_rng(100 + call)
-        host = [np.zeros((g.n, ld), np.float32) for _ in range(4)]
+        host = [np.full((g.n, ld), 2.5, np.float32) for _ in range(4)]        # padding columns: never used
         host[0][:, :N] = 0.3 * rng.standard_normal((g.n, N))
         host[1][:, :N] = 0.05 * rng.standard_normal((g.n, N))
         host[2][:, :N] = rng.uniform(0.5, 2.0, (g.n, N))
         host[3][:, :N] = rng.standard_normal((g.n, N))
         arrays = [torch.from_numpy(h).cuda() for h in host]
         want = _reference_scales(torch, B, g, N, ld, kind, bits, arrays, sigma, noise, gamma, seed, call)
+        oracle = _oracle_scales(g, N, kind, bits, host, sigma, noise, gamma, seed, call)
         before = [t.clone() for t in arrays]
         out.fill_(-1.0)
         st = B.ds_node_scales_noalloc(out, arrays[0], arrays[1], arrays[2], arrays[3], sigma, noise,
@@ -55,7 +81,8 @@ def test_noalloc_scales_match_regular_path_twice(kind, bits):
         torch.cuda.synchronize()
         got = out.cpu().numpy()
         assert np.all(got > 0)
-        assert np.abs(got - want).max() <= TOL * np.abs(want).max(), (got, want)
+        _assert_scales(kind, got, want, "against ds_step with chunk = 0")
+        _assert_scales(kind, got, oracle, "against the CPU oracle")
         for t, b in zip(arrays, before):          # inputs are only read
             assert torch.equal(t, b)
 
