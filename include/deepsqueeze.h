@@ -21,7 +21,12 @@
  *     Columns N..ld-1 are padding: read, never changed.
  *   - Pointers are DEVICE pointers unless the comment says "host".
  *   - The caller owns every buffer, the workspace included; the library
- *     allocates no device memory.  x and delta are updated in place.
+ *     calls no device-memory allocator (cudaMalloc and friends).  x and delta
+ *     are updated in place.  Two entry points create other driver objects
+ *     inside the context, on first use, and ds_destroy releases them:
+ *     ds_run records and instantiates a CUDA graph (one internal capture
+ *     stream, one executable graph), ds_step_host creates three streams and
+ *     34 events for its copy/compute pipeline.  Nothing else creates any.
  *   - Every call returns a ds_status; nothing throws.  ds_step only enqueues
  *     work on the given stream and reports argument and launch errors.
  *   - One ds_ctx must not be used from two streams at once (the steps share
@@ -78,7 +83,9 @@ typedef struct {
  *                                Euclidean norm ||v||_2, and the receiver rescales what it
  *                                decodes to that norm: C = level[code] * ||v||_2 / ||level[code]||_2.
  *                                Deterministic and biased -- what error compensation is for.
- *                                chunk must be in 32..512 (one chunk = one "tensor").
+ *                                One chunk = one "tensor"; chunk = 0 is the paper's granularity,
+ *                                one norm for the node's whole vector (two more reduction
+ *                                launches per step: the maximum, then the two sums of squares).
  * chunk: elements per scale, a multiple of 32; 0 = one scale per node. */
 typedef enum {
     DS_COMP_IDENTITY = 0,
@@ -149,7 +156,9 @@ typedef struct {
 } ds_info;
 
 /* Bytes of device workspace ds_init needs for this shape (host-only call;
- * returns 0 for invalid arguments).  nnz = row_ptr[n]. */
+ * returns 0 for invalid arguments).  nnz = row_ptr[n]: the workspace also holds
+ * the CSR of W - I and of W (what ds_init validates and copies), so its size
+ * depends on the number of edges -- the one argument beyond (n, N, compressor). */
 size_t ds_workspace_size(int32_t n, int64_t N, const ds_compressor *comp, int32_t nnz);
 
 /* Validate the graph and W (Assumption 1: W symmetric, doubly stochastic;
@@ -264,7 +273,12 @@ ds_status ds_run_resident(ds_ctx *ctx, float *x, float *delta, const ds_grad_par
  * column tiles and pipelined on three internal streams (created at the first
  * call): while one slab is computed the next is on its way in and the previous
  * on its way out.  Padding columns are copied in, never out.  dev_* are device
- * [n][ld] arrays owned by the caller.  Only the synthetic objective. */
+ * [n][ld] arrays owned by the caller.  Only the synthetic objective.
+ * Not pipelined (four whole-array copies in, one step, two copies out, all on
+ * `cuda_stream`): arrays below 64 MiB, one scale per node, and the case that the
+ * internal streams or events cannot be created.  If a call fails after work
+ * has been enqueued on the internal streams, that work is joined into
+ * `cuda_stream` before the error status is returned. */
 ds_status ds_step_host(ds_ctx *ctx, float *x_host, float *delta_host,
                        const float *a_host, const float *c_host,
                        float sigma, int32_t noise, const ds_hparams *hp,

@@ -159,7 +159,11 @@ def ds_init_raw(row_ptr, col_idx, w, n: int, N: int, ld: int, kind: int, bits: i
 class DeepSqueeze:
     """A context plus the workspace tensor that backs it (torch owns the memory)."""
 
-    def __init__(self, graph, N: int, ld: int, kind: int, bits: int, chunk: int, device="cuda:0"):
+    def __init__(self, graph, N: int, ld: int, kind: int, bits: int, chunk: int, device="cuda:0",
+                 guard_bytes: int = 0):
+        """guard_bytes > 0 (a multiple of 256) puts that many bytes of a fixed pattern directly
+        before and after the workspace; workspace_guards_intact() tells whether any of them
+        changed -- a bounds check for kernels that write into the workspace."""
         import torch
         self.torch = torch
         self.n, self.N, self.ld = graph.n, int(N), int(ld)
@@ -169,14 +173,24 @@ class DeepSqueeze:
         size = ds_workspace_size(self.n, self.N, kind, bits, chunk, nnz)
         if size == 0:
             raise DsError(DS_ERR_UNSUPPORTED, "ds_workspace_size")
+        assert guard_bytes >= 0 and guard_bytes % 256 == 0
+        self.guard_bytes, self.ws_bytes = guard_bytes, size
         with torch.cuda.device(self.device):
-            self.workspace = torch.empty(size + 256, dtype=torch.uint8, device=self.device)
-            ptr = (self.workspace.data_ptr() + 255) // 256 * 256
+            self.workspace = torch.full((size + 256 + 2 * guard_bytes,), 0xA5, dtype=torch.uint8, device=self.device)
+            ptr = (self.workspace.data_ptr() + 255) // 256 * 256 + guard_bytes
+            self.ws_ptr = ptr
             st, ctx = ds_init_raw(graph.row_ptr, graph.col_idx, graph.w, self.n, self.N, self.ld,
                                   kind, bits, chunk, ptr, size)
         _check(st, "ds_init")
         self.ctx = ctx
         self.code_bits = 32 if kind == DS_COMP_IDENTITY else (1 if kind == DS_COMP_SIGN1_L1 else bits)
+
+    def workspace_guards_intact(self) -> bool:
+        """True if the pattern bytes before and after the workspace are all unchanged."""
+        off = self.ws_ptr - self.workspace.data_ptr()
+        front = self.workspace[off - self.guard_bytes: off]
+        back = self.workspace[off + self.ws_bytes: off + self.ws_bytes + self.guard_bytes]
+        return bool((front == 0xA5).all()) and bool((back == 0xA5).all())
 
     def ds_set_path(self, path: int):
         _check(lib().ds_set_path(self.ctx, path), "ds_set_path")
@@ -294,7 +308,7 @@ class DeepSqueeze:
         """Copy the last step's packed codes [n][words] and scales [n][M] to numpy."""
         torch = self.torch
         cptr, cpitch, sptr, spitch = self.ds_codes()
-        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        base = self.ws_ptr
         ws = self.workspace[base - self.workspace.data_ptr():]
         words = (self.N * self.code_bits + 31) // 32
         codes = ws[cptr - base: cptr - base + self.n * cpitch * 4].view(torch.int32).view(self.n, cpitch)

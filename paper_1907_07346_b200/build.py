@@ -19,7 +19,8 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdeepsqueeze.so")
 SOURCES = ["ds_api.cu", "ds_kernels_tma.cu", "ds_kernels_fused.cu", "ds_kernels_wide.cu", "ds_kernels_wide_tma.cu", "ds_kernels_compress.cu",
-           "ds_kernels_misc.cu", "ds_noalloc.cu", "ds_kernels_resident.cu", "ds_kernels_tma_pair.cu", "ds_kernels_tma_ecsgd.cu"]
+           "ds_kernels_misc.cu", "ds_noalloc.cu", "ds_kernels_resident.cu", "ds_kernels_tma_pair.cu", "ds_kernels_tma_ecsgd.cu",
+           "ds_kernels_wide_norm.cu", "ds_kernels_wide_tma_norm.cu", "ds_kernels_reduce_norm.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-fmad=false", "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
 

@@ -38,7 +38,7 @@ struct Shape {
 };
 
 struct WsLayout {
-    size_t codes, scales, dscales, partials, rpartials, row_ptr, col_idx, wprime, wplain, lut, error_flag, barrier, total;
+    size_t codes, scales, dscales, partials, gmax, rpartials, row_ptr, col_idx, wprime, wplain, lut, error_flag, barrier, total;
 };
 
 bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
@@ -57,11 +57,11 @@ bool make_shape(int32_t n, int64_t N, const ds_compressor* comp, Shape* sh) {
             else return false;
             break;
         case DS_COMP_UNIFORM_NEAREST_L2:
-            // the paper's own settings (2 and 4 bits); one warp codes a chunk, so chunk <= 512
+            // the paper's own settings (2 and 4 bits); any chunk, or chunk = 0: one norm per node,
+            // the paper's "one Euclidean norm per tensor"
             if (comp->bits == 2) sh->code = CODE_N2;
             else if (comp->bits == 4) sh->code = CODE_N4;
             else return false;
-            if (comp->chunk < 32 || comp->chunk > 512) return false;
             break;
         default: return false;
     }
@@ -95,7 +95,9 @@ WsLayout make_ws(int32_t n, int32_t nnz, const Shape& sh) {
     const bool norm = (sh.code == CODE_N2 || sh.code == CODE_N4);
     w.dscales = norm ? off : w.scales;      // decode factors only differ from the sent scalars for norm-matched codes
     if (norm) off = align_up(off + (size_t)n * (size_t)sh.scales_pitch * 4, kAlign);
-    w.partials = off; off = align_up(off + (sh.per_node ? (size_t)n * (size_t)sh.tiles * 8 : 0), kAlign);
+    // per-node scale: one binary64 partial per (node, tile); a per-node norm needs two sums
+    w.partials = off; off = align_up(off + (sh.per_node ? (norm ? 2 : 1) * (size_t)n * (size_t)sh.tiles * 8 : 0), kAlign);
+    w.gmax = off;     off = align_up(off + (sh.per_node && norm ? (size_t)n * 4 : 0), kAlign);
     // two buffers of per-tile partials for the resident multi-step kernel (small per-node-scale shapes only)
     w.rpartials = off;
     off = align_up(off + (resident_shape(n, sh) && sh.per_node ? 2 * (size_t)n * (size_t)sh.tiles * 8 : 0), kAlign);
@@ -131,7 +133,6 @@ Plan plan_column(int mode, const Shape& sh, int32_t n, int32_t nnz, int force_e 
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
     if (G > 32) return pl;
-    if ((sh.code == CODE_N2 || sh.code == CODE_N4) && G != 1) return pl;
     int npb;
     if (mode == MODE_FUSED) {
         if (sh.code == CODE_ID32) return pl;
@@ -158,7 +159,6 @@ Plan plan_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int force_e 
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
     if ((int64_t)n * G > 32 || num_sms < 1) return pl;
-    if ((sh.code == CODE_N2 || sh.code == CODE_N4) && G != 1) return pl;
     // every warp of a group owns a whole E*32-element segment
     if ((int64_t)G * E * 32 < sh.tile) return pl;
     pl.nodes_per_block = n;
@@ -195,7 +195,7 @@ Plan plan_wide(const Shape& sh, int32_t n, int32_t nnz, int force_e = 0) {
     pick_lane_shape(sh.tile, force_e, &E, &G);
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
-    if (sh.code == CODE_ID32 || sh.code == CODE_N2 || sh.code == CODE_N4 || G > 16) return pl;
+    if (sh.code == CODE_ID32 || G > 16) return pl;
     const int npb = std::max(1, std::min<int>(n, 16 / G));
     pl.nodes_per_block = npb;
     pl.block = dim3((unsigned)(npb * G * 32));
@@ -214,7 +214,7 @@ Plan plan_wide_tma(const Shape& sh, int32_t n, int32_t nnz, int num_sms, int for
     pick_lane_shape(sh.tile, force_e, &E, &G);
     pl.elems_per_lane = E;
     pl.warps_per_group = G;
-    if (sh.code == CODE_ID32 || sh.code == CODE_N2 || sh.code == CODE_N4 || E < 8 || G > 16 || num_sms < 1) return pl;
+    if (sh.code == CODE_ID32 || E < 8 || G > 16 || num_sms < 1) return pl;
     const int npb = std::max(1, std::min<int>(n, 16 / G));
     pl.nodes_per_block = npb;
     pl.block = dim3((unsigned)(npb * G * 32));
@@ -444,7 +444,8 @@ ds_status ds_get_info(const ds_ctx* ctx, ds_info* info) {
                    : (kind == 3) ? ctx->wide : ctx->compress;
     info->path = (kind == 2 || kind == 4 || kind == 5) ? DS_PATH_FUSED : (kind != 0) ? DS_PATH_FUSED_LDG : DS_PATH_SPLIT;
     info->node_batches = (kind == 3 || kind == 4) ? (ctx->n + pl.nodes_per_block - 1) / pl.nodes_per_block : 1;
-    info->launches_per_step = (fused ? 1 : 2) + (ctx->sh.per_node ? 2 : 0);
+    const bool norm = (ctx->sh.code == CODE_N2 || ctx->sh.code == CODE_N4);
+    info->launches_per_step = (fused ? 1 : 2) + (ctx->sh.per_node ? (norm ? 4 : 2) : 0);
     info->elems_per_lane = pl.elems_per_lane;
     info->warps_per_chunk = pl.warps_per_group;
     info->block_threads = (int32_t)pl.block.x;
@@ -496,6 +497,8 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
     p.scales_pitch = ctx->sh.scales_pitch;
     p.dscales = reinterpret_cast<float*>(ctx->base + ctx->ws.dscales);
     p.partials = reinterpret_cast<double*>(ctx->base + ctx->ws.partials);
+    p.gmax = reinterpret_cast<float*>(ctx->base + ctx->ws.gmax);
+    p.norm_phase = 0;
     p.error_flag = reinterpret_cast<int*>(ctx->base + ctx->ws.error_flag);
     p.sigma = sigma;
     p.neg_gamma = -hp->gamma;
@@ -522,6 +525,14 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
         p.nodes_per_block = ctx->reduce.nodes_per_block;
         e = launch_column_reduce(shape_of(ctx->reduce, MODE_REDUCE), p, stream);
         if (e == cudaSuccess) e = launch_finalize_scales(p, ctx->sh.code, stream);
+        if (ctx->sh.code == CODE_N2 || ctx->sh.code == CODE_N4) {
+            // one norm per node (Section 5: one Euclidean norm per tensor): with the maximum
+            // known, a second reduction takes the sums of v^2 and of level^2
+            p.norm_phase = 2;
+            if (e == cudaSuccess) e = launch_column_reduce_norm(shape_of(ctx->reduce, MODE_REDUCE), p, stream);
+            if (e == cudaSuccess) e = launch_finalize_norms(p, stream);
+            p.norm_phase = 0;
+        }
     }
     if (e == cudaSuccess) {
         // centralized error-compensated SGD: the fused kernel where the shape allows
@@ -690,6 +701,8 @@ ds_status ds_run_resident(ds_ctx* ctx, float* x, float* delta, const ds_grad_par
     p.scales_pitch = ctx->sh.scales_pitch;
     p.dscales = reinterpret_cast<float*>(ctx->base + ctx->ws.dscales);
     p.partials = reinterpret_cast<double*>(ctx->base + ctx->ws.partials);
+    p.gmax = nullptr;
+    p.norm_phase = 0;
     p.error_flag = reinterpret_cast<int*>(ctx->base + ctx->ws.error_flag);
     p.sigma = gp->sigma;
     p.neg_gamma = 0.0f; p.eta = 0.0f;

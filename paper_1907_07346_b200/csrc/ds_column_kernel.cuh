@@ -38,8 +38,8 @@ __host__ __device__ inline SmemLayout smem_layout(int mode, int code_bits, bool 
     SmemLayout L;
     uint32_t off = 0;
     L.cw = (uint32_t)((tile * code_bits + 31) / 32);
-    L.red_off = off;
-    off += (G > 1) ? (uint32_t)(npb * G) * 8u : 0u;
+    L.red_off = off;                      // three binary64 slots per warp: scale partial, two norm sums
+    off += (G > 1) ? 3u * (uint32_t)(npb * G) * 8u : 0u;
     L.codes_off = off;
     off += (mode == MODE_FUSED) ? 2u * (uint32_t)npb * L.cw * 4u : 0u;
     L.scale_off = off;
@@ -81,20 +81,21 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
-// Norm-matched b-bit compression of one chunk held by ONE warp (Section 5,
-// "Compression": b bits per element plus the Euclidean norm of the tensor; the
-// receiver rescales what it decodes to that norm).
+// Norm-matched b-bit compression (Section 5, "Compression": b bits per element
+// plus the Euclidean norm of the tensor; the receiver rescales what it decodes
+// to that norm), in two halves so that a chunk may be spread over several warps
+// or, with one norm per node, over several launches:
 //   m = max |v| spans the grid; code = clamp(floor(fma(v/m, L/2, L/2) + 1/2), 0, L)
-//   (round to nearest level); l_k = level[code_k];
+//   (round to nearest level); l_k = level[code];
 //   nrm = sqrt(sum v_k^2), lnorm = sqrt(sum l_k^2) (binary64 sums, rounded to binary32);
 //   r = nrm / lnorm;  C_k = r * l_k.
-// A lane holds E elements, element 4*(32*r + lane) + j of the chunk at index
-// 4*r + j; only the first valid_len elements of the chunk count.  On return
-// q[] holds the codes, cv[] the C values, nrm the scalar to send and r the
-// decode factor.  m = 0 or not finite: codes 0, nrm = r = 0.
-template <int CODE, int E, bool FULL>
-__device__ __forceinline__ void norm_compress(const float* v, int valid_len, float m, const float* lut,
-                                              int lane, uint32_t* q, float* cv, float& nrm, float& r) {
+// norm_codes(): codes and levels of the E elements a lane holds, and the two
+// binary64 sums over the WARP's valid elements (lane order, then a butterfly);
+// valid(t) tells whether the lane's element t counts.  m = 0 or not finite:
+// codes 0.  The caller adds up the sums of the chunk's warps in warp order.
+template <int CODE, int E, bool FULL, class ValidFn>
+__device__ __forceinline__ void norm_codes(const float* v, ValidFn valid, float m, const float* lut,
+                                           uint32_t* q, float* lv, double& sv2_out, double& sl2_out) {
     constexpr int kBits = (CODE == CODE_N2) ? 2 : 4;
     constexpr int kLi = (1 << kBits) - 1;
     constexpr float kHalfL = 0.5f * (float)kLi;
@@ -107,8 +108,7 @@ __device__ __forceinline__ void norm_compress(const float* v, int valid_len, flo
     const double* lut_sq = reinterpret_cast<const double*>(lut + 32);
 #pragma unroll
     for (int t = 0; t < E; ++t) {
-        const int k = 4 * (32 * (t >> 2) + lane) + (t & 3);
-        const bool ok = FULL || k < valid_len;
+        const bool ok = FULL || valid(t);
         float y;
         if (fast) {
             const float q0 = __fmul_rn(v[t], inv);
@@ -120,7 +120,7 @@ __device__ __forceinline__ void norm_compress(const float* v, int valid_len, flo
         const float u = __fmaf_rn(y, kHalfL, kHalfL);
         const uint32_t code = dead ? 0u : (uint32_t)min(max(__float2int_rd(__fadd_rn(u, 0.5f)), 0), kLi);
         q[t] = code;
-        cv[t] = lut[code];
+        lv[t] = lut[code];
         if (ok) {
             // products of two binary32 numbers are exact in binary64, so the fused
             // form rounds exactly like "sum += product"
@@ -133,13 +133,25 @@ __device__ __forceinline__ void norm_compress(const float* v, int valid_len, flo
         sv2 += __shfl_xor_sync(0xffffffffu, sv2, o);
         sl2 += __shfl_xor_sync(0xffffffffu, sl2, o);
     }
+    sv2_out = sv2;
+    sl2_out = sl2;
+}
+
+// norm_finish(): from the two sums of the whole chunk the scalar that is sent
+// (nrm) and the factor the receiver applies to the levels (r).  m = 0 or not
+// finite, or a norm that is not finite: nrm = r = 0.
+__device__ __forceinline__ void norm_finish(float m, double sv2, double sl2, float& nrm, float& r) {
+    const bool dead = (m == 0.0f) || !(m <= 3.402823466e+38f);
     nrm = dead ? 0.0f : (float)sqrt(sv2);
     const float lnorm = (float)sqrt(sl2);
     r = (dead || lnorm == 0.0f || !(nrm <= 3.402823466e+38f)) ? 0.0f : __fdiv_rn(nrm, lnorm);
     if (!(nrm <= 3.402823466e+38f)) nrm = 0.0f;
-#pragma unroll
-    for (int t = 0; t < E; ++t) cv[t] = __fmul_rn(r, cv[t]);
 }
+
+// The factor a receiver multiplies the levels by: the scale that is sent, except for
+// norm-matched codes, where the sent scalar is the norm and the factor norm / ||levels||.
+template <bool NORM>
+__device__ __forceinline__ float dscale_of(float sent, float factor) { return NORM ? factor : sent; }
 
 __device__ __forceinline__ float4 ld4(const float* p) {
     return __ldcs(reinterpret_cast<const float4*>(p));
@@ -211,9 +223,14 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
 
     // ---------------- scale of the (node, tile) --------------------------
     float s = 1.0f;
+    // norm-matched codes with one norm per node take two reductions: the maximum that spans
+    // the grid (norm_phase 0, like every per-node scale), then, with the maximum known, the two
+    // sums of squares (norm_phase 2)
+    const bool norm_sums_pass = T::kNorm && MODE == MODE_REDUCE && p.norm_phase == 2;
     if constexpr (!T::kIdentity) {
-        if (p.prescaled && MODE != MODE_REDUCE) {
-            s = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+        if (p.prescaled && (MODE != MODE_REDUCE || norm_sums_pass)) {
+            if constexpr (T::kNorm) s = node_ok ? p.gmax[node] : 0.0f;
+            else s = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
         } else {
             double part;
             if constexpr (T::kSign) part = warp_sum(sum);
@@ -243,7 +260,7 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
             }
         }
     }
-    if constexpr (MODE == MODE_REDUCE) return;
+    if constexpr (MODE == MODE_REDUCE && !T::kNorm) return;
     const bool degenerate = (!T::kSign && !T::kIdentity && s == 0.0f);
     // the quotient v/s may use the reciprocal only while s is far from the
     // ends of the exponent range (uniform over the group)
@@ -256,16 +273,45 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
     const size_t code_row = (size_t)node * (size_t)p.code_pitch
                           + (size_t)((k0 * T::kBits) >> 5);
 
-    // norm-matched codes (one warp per chunk only): code the whole chunk first;
-    // s becomes the norm that is sent, dscale the factor the receiver applies
+    // norm-matched codes: code the whole chunk first; s becomes the norm that is sent,
+    // dscale the factor the receiver applies
     uint32_t qn[T::kNorm ? E : 1];
     float cvn[T::kNorm ? E : 1];
     float dscale = s;
     if constexpr (T::kNorm) {
+        auto valid = [&](int t) { return node_ok && 4 * (f0 + fstride * (t >> 2)) + (t & 3) < m_len; };
+        double sv2, sl2;
+        norm_codes<CODE, E, FULL>(v, valid, s, lut, qn, cvn, sv2, sl2);
         float nrm;
-        norm_compress<CODE, E, FULL>(v, node_ok ? m_len : 0, s, lut, lane, qn, cvn, nrm, dscale);
+        if (p.prescaled && MODE != MODE_REDUCE) {
+            // one norm per node, computed by the earlier launches
+            nrm = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+            dscale = node_ok ? p.dscales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+        } else {
+            if (G > 1) {
+                // the sums of the chunk's warps, added in warp order
+                double* red2 = reinterpret_cast<double*>(smem + L.red_off) + (size_t)p.nodes_per_block * G;
+                double* red3 = red2 + (size_t)p.nodes_per_block * G;
+                if (lane == 0) { red2[grp * G + wg] = sv2; red3[grp * G + wg] = sl2; }
+                __syncthreads();
+                sv2 = 0.0; sl2 = 0.0;
+                for (int w = 0; w < G; ++w) { sv2 += red2[grp * G + w]; sl2 += red3[grp * G + w]; }
+                if (MODE == MODE_REDUCE) __syncthreads();      // the slots are written again for the next tile
+            }
+            if constexpr (MODE == MODE_REDUCE) {
+                if (node_ok && wg == 0 && lane == 0) {
+                    p.partials[(size_t)node * (size_t)p.tiles + (size_t)col] = sv2;
+                    p.partials[((size_t)p.n + (size_t)node) * (size_t)p.tiles + (size_t)col] = sl2;
+                }
+                return;
+            }
+            norm_finish(s, sv2, sl2, nrm, dscale);
+        }
+#pragma unroll
+        for (int t = 0; t < E; ++t) cvn[t] = __fmul_rn(dscale, cvn[t]);
         s = nrm;
     }
+    if constexpr (MODE == MODE_REDUCE) return;
 
     // ---------------- phase B: compress, residual, pack ------------------
     constexpr float kL = (float)((1u << (T::kBits & 15)) - 1u);

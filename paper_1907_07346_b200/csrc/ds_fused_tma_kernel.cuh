@@ -45,7 +45,7 @@ __host__ __device__ inline TmaSmemLayout tma_smem_layout(bool has_lut, int E, in
     L.seg_bytes = (uint32_t)E * 32u * 4u;
     L.slots_off = off;   off += (uint32_t)nwarps * 4u * L.seg_bytes;
     L.cval_off = off;    off += 2u * (uint32_t)n * (uint32_t)tile * 4u;
-    L.red_off = off;     off += (G > 1) ? (uint32_t)nwarps * 8u : 0u;
+    L.red_off = off;     off += (G > 1) ? 3u * (uint32_t)nwarps * 8u : 0u;   // scale partial and two norm sums per warp
     L.mbar_off = off;    off += (uint32_t)nwarps * 8u;
     L.nbar_off = off;    off += 2u * (uint32_t)n * 8u;      // "C[v] of node j is ready", one per buffer and node
     L.lut_off = off;     off += has_lut ? 256u * 4u : 0u;
@@ -191,13 +191,16 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     // the rounding uniforms of the stochastic quantiser are drawn with it
     constexpr bool kRndAhead = T::kLut && !T::kNorm;
     float mn[kRndAhead ? E : 1];
-    auto draw_noise = [&](int64_t c) {
+    // do_noise / do_rnd select which of the two streams are drawn by this call
+    auto draw_noise = [&](int64_t c, auto noise_tag, auto rnd_tag) {
+        constexpr bool DO_NOISE = decltype(noise_tag)::value && kNoiseAhead;
+        constexpr bool DO_RND = decltype(rnd_tag)::value && kRndAhead;
         const uint32_t kbase = (uint32_t)(c * p.tile + seg0) + 4u * (uint32_t)lane;   // element of r = 0
-        if constexpr (kNoiseAhead || kRndAhead) {
-            // all Philox blocks of the tile (V for the noise, V for the rounding stream,
-            // whichever are needed) advance together
-            constexpr int kGauss = kNoiseAhead ? V : 0;
-            constexpr int kRnd = kRndAhead ? V : 0;
+        if constexpr (DO_NOISE || DO_RND) {
+            // all Philox blocks of the call (V for the noise, V for the rounding stream,
+            // whichever are drawn) advance together
+            constexpr int kGauss = DO_NOISE ? V : 0;
+            constexpr int kRnd = DO_RND ? V : 0;
             uint32_t stream[kGauss + kRnd], block[kGauss + kRnd];
             uint4 w[kGauss + kRnd];
 #pragma unroll
@@ -220,7 +223,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             }
         }
     };
-    if (col < p.tile_end) draw_noise(col);      // (also when only the rounding stream is needed)
+    if (col < p.tile_end) draw_noise(col, std::true_type{}, std::true_type{});      // (also when only the rounding stream is needed)
     uint32_t parity = 0;
     int buf = 0;
     uint32_t iter = 0;          // tiles this block has worked on
@@ -230,8 +233,11 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
 
     for (; col < p.tile_end; col += gridDim.x, ++iter) {
         if (drain) {
-            // (the block-wide barrier of the scale reduction of a multi-warp chunk is still kept)
-            if (G > 1 && !T::kIdentity && !p.prescaled) __syncthreads();
+            // (the block-wide barriers of the reductions of a multi-warp chunk are still kept)
+            if (G > 1 && !T::kIdentity && !p.prescaled) {
+                __syncthreads();
+                if constexpr (T::kNorm) __syncthreads();
+            }
             if (lane == 0) mbar_arrive(nbar0 + 8u * (uint32_t)(buf * p.n + node));
             buf ^= 1;
             continue;
@@ -305,7 +311,8 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             if constexpr (T::kIdentity) {
                 s = 1.0f;                       // C[v] = v: nothing to scale
             } else if (p.prescaled) {
-                s = p.scales[(size_t)node * (size_t)p.scales_pitch];
+                if constexpr (T::kNorm) s = p.gmax[node];          // the maximum that spans the grid
+                else s = p.scales[(size_t)node * (size_t)p.scales_pitch];
             } else {
                 double part;
                 if constexpr (T::kSign) part = warp_sum(sum);
@@ -344,8 +351,28 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             float cvn[T::kNorm ? E : 1];
             float dscale = s;
             if constexpr (T::kNorm) {
+                auto valid = [&](int t) { return 4 * (32 * (t >> 2) + lane) + (t & 3) < live_len; };
+                double sv2, sl2;
+                norm_codes<CODE, E, FULL>(v, valid, s, lut, qn, cvn, sv2, sl2);
                 float nrm;
-                norm_compress<CODE, E, FULL>(v, live_len, s, lut, lane, qn, cvn, nrm, dscale);
+                if (p.prescaled) {
+                    // one norm per node, computed by the earlier launches
+                    nrm = p.scales[(size_t)node * (size_t)p.scales_pitch];
+                    dscale = p.dscales[(size_t)node * (size_t)p.scales_pitch];
+                } else {
+                    if (G > 1) {
+                        // the sums of the chunk's warps, added in warp order
+                        double* red2 = reinterpret_cast<double*>(smem + L.red_off) + nwarps;
+                        double* red3 = red2 + nwarps;
+                        if (lane == 0) { red2[warp] = sv2; red3[warp] = sl2; }
+                        __syncthreads();
+                        sv2 = 0.0; sl2 = 0.0;
+                        for (int w = 0; w < G; ++w) { sv2 += red2[node * G + w]; sl2 += red3[node * G + w]; }
+                    }
+                    norm_finish(s, sv2, sl2, nrm, dscale);
+                }
+    #pragma unroll
+                for (int t = 0; t < E; ++t) cvn[t] = __fmul_rn(dscale, cvn[t]);
                 s = nrm;
             }
 
@@ -426,6 +453,11 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             // before it is written again two tiles later.)
             __syncwarp();
             if (lane == 0) mbar_arrive(nbar0 + 8u * (uint32_t)(buf * p.n + node));
+            // The gradient noise of the next tile needs nothing from the neighbours: it is drawn
+            // HERE, between the announcement and the wait, so that by the time this warp looks at
+            // its neighbours' barriers they have normally completed and it does not poll.
+            const bool more = col + gridDim.x < p.tile_end;
+            if (more) draw_noise(col + gridDim.x, std::true_type{}, std::false_type{});
             {
                 const uint32_t nphase = (iter >> 1) & 1u;
                 bool ok = true;
@@ -472,7 +504,8 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     st_partial(x_lane + 128 * r, make_float4(xa.x, xa.y, xb.x, xb.y), nv);
                 }
             }
-            if (col + gridDim.x < p.tile_end) draw_noise(col + gridDim.x);
+            // (the rounding uniforms of the next tile after the mix, when fewer registers are live)
+            if (more) draw_noise(col + gridDim.x, std::false_type{}, std::true_type{});
             return false;
         };
         const bool aborted = full ? tile_body(std::true_type{}) : tile_body(std::false_type{});

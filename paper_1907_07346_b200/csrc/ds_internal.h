@@ -41,7 +41,9 @@ struct StepParams {
     int64_t scales_pitch;
     float* dscales;           // the factor the receiver multiplies the levels by (= scales unless the
                               // decoder rescales to a norm), same pitch
-    double* partials;         // [n][tiles], per-node-scale reduction
+    double* partials;         // [n][tiles], per-node-scale reduction (twice that for the two sums of a
+                              // per-node norm: sum v^2 in the first half, sum level^2 in the second)
+    float* gmax;              // [n], norm-matched codes with one norm per node: max |v| of the node
     int* error_flag;          // set to 1 by a kernel whose bounded wait ran out
     float sigma;
     float neg_gamma;
@@ -50,6 +52,7 @@ struct StepParams {
     int32_t warps_per_group;  // warps sharing one (node, tile)
     int32_t nodes_per_block;
     int32_t prescaled;        // 1: scale of node i is scales[i][0], computed by an earlier launch
+    int32_t norm_phase;       // reduce mode, norm-matched codes, one norm per node: 0 = maximum, 2 = sums of squares
     int32_t ecsgd;            // 1 (compress / reduce modes only): centralized error-compensated SGD,
                               // v = g + delta is compressed and x is left for the server's update
 };
@@ -69,9 +72,13 @@ cudaError_t launch_column_fused(const LaunchShape& shape, const StepParams& p, c
 cudaError_t launch_fused_tma(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_fused_wide_tma(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_fused_wide(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
+cudaError_t launch_fused_wide_tma_norm(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
+cudaError_t launch_fused_wide_norm(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_column_compress(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
 cudaError_t launch_column_reduce(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
-cudaError_t launch_finalize_scales(const StepParams& p, int code, cudaStream_t stream);
+cudaError_t launch_column_reduce_norm(const LaunchShape& shape, const StepParams& p, cudaStream_t stream);
+cudaError_t launch_finalize_scales(const StepParams& p, int code, cudaStream_t stream);   // norm-matched codes: the maximum, into gmax
+cudaError_t launch_finalize_norms(const StepParams& p, cudaStream_t stream);
 cudaError_t launch_mix_kernel(const StepParams& p, int code, cudaStream_t stream);
 cudaError_t launch_math_selftest(unsigned long long* counts, cudaStream_t stream);
 cudaError_t launch_wait_selftest(int* error_flag, cudaStream_t stream);

@@ -96,7 +96,8 @@ cudaError_t launch_mix_kernel(const StepParams& p, int code, cudaStream_t stream
 // One warp per node.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(32) ds_finalize_scales_kernel(const __grid_constant__ StepParams p,
-                                                                const int sign) {
+                                                                const int sign, float* const out,
+                                                                const int64_t out_pitch) {
     const int node = blockIdx.x;
     const int lane = threadIdx.x;
     const double* part = p.partials + (size_t)node * (size_t)p.tiles;
@@ -115,12 +116,47 @@ __global__ void __launch_bounds__(32) ds_finalize_scales_kernel(const __grid_con
             s = (float)acc;
             if (s == 0.0f || !(fabsf(s) <= 3.402823466e+38f)) s = 0.0f;
         }
-        p.scales[(size_t)node * (size_t)p.scales_pitch] = s;
+        out[(size_t)node * (size_t)out_pitch] = s;
     }
 }
 
 cudaError_t launch_finalize_scales(const StepParams& p, int code, cudaStream_t stream) {
-    ds_finalize_scales_kernel<<<p.n, 32, 0, stream>>>(p, code == CODE_SIGN ? 1 : 0);
+    // norm-matched codes: this maximum only spans the grid; it goes to gmax, the norms follow
+    const bool norm = (code == CODE_N2 || code == CODE_N4);
+    ds_finalize_scales_kernel<<<p.n, 32, 0, stream>>>(p, code == CODE_SIGN ? 1 : 0, norm ? p.gmax : p.scales,
+                                                      norm ? 1 : p.scales_pitch);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------
+// Norm-matched codes, one norm per node (Section 5, "Compression": b bits per
+// element plus the Euclidean norm of the tensor): combine the per-tile sums of
+// v^2 (first half of the partials) and of level^2 (second half) of one node in
+// the same fixed order as above; write the norm that is sent and the factor
+// norm / ||levels|| the receivers apply.  One warp per node.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(32) ds_finalize_norms_kernel(const __grid_constant__ StepParams p) {
+    const int node = blockIdx.x;
+    const int lane = threadIdx.x;
+    const double* pv = p.partials + (size_t)node * (size_t)p.tiles;
+    const double* pl = p.partials + ((size_t)p.n + (size_t)node) * (size_t)p.tiles;
+    double sv2 = 0.0, sl2 = 0.0;
+    for (int64_t t = lane; t < p.tiles; t += 32) { sv2 += pv[t]; sl2 += pl[t]; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        sv2 += __shfl_xor_sync(0xffffffffu, sv2, o);
+        sl2 += __shfl_xor_sync(0xffffffffu, sl2, o);
+    }
+    if (lane == 0) {
+        float nrm, r;
+        norm_finish(p.gmax[node], sv2, sl2, nrm, r);
+        p.scales[(size_t)node * (size_t)p.scales_pitch] = nrm;
+        p.dscales[(size_t)node * (size_t)p.scales_pitch] = r;
+    }
+}
+
+cudaError_t launch_finalize_norms(const StepParams& p, cudaStream_t stream) {
+    ds_finalize_norms_kernel<<<p.n, 32, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

@@ -10,6 +10,7 @@ cudaError_t launch_fused_wide(const LaunchShape& sh, const StepParams& p, cudaSt
         case CODE_U2: return launch_wide_code<CODE_U2>(sh, p, stream);
         case CODE_U4: return launch_wide_code<CODE_U4>(sh, p, stream);
         case CODE_U8: return launch_wide_code<CODE_U8>(sh, p, stream);
+        case CODE_N2: case CODE_N4: return launch_fused_wide_norm(sh, p, stream);
         default: return cudaErrorInvalidValue;
     }
 }

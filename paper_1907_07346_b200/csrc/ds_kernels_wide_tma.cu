@@ -10,6 +10,7 @@ cudaError_t launch_fused_wide_tma(const LaunchShape& sh, const StepParams& p, cu
         case CODE_U2: return launch_wide_tma_code<CODE_U2>(sh, p, stream);
         case CODE_U4: return launch_wide_tma_code<CODE_U4>(sh, p, stream);
         case CODE_U8: return launch_wide_tma_code<CODE_U8>(sh, p, stream);
+        case CODE_N2: case CODE_N4: return launch_fused_wide_tma_norm(sh, p, stream);
         default: return cudaErrorInvalidValue;
     }
 }

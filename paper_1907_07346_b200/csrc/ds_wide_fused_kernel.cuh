@@ -29,7 +29,7 @@ __host__ __device__ inline WideSmemLayout wide_smem_layout(int code_bits, bool h
     WideSmemLayout L;
     uint32_t off = 0;
     L.cw = (uint32_t)((tile * code_bits + 31) / 32);
-    L.red_off = off;     off += 2u * (uint32_t)(npb * G) * 8u;
+    L.red_off = off;     off += 2u * 3u * (uint32_t)(npb * G) * 8u;   // two alternating sets of (scale partial, two norm sums)
     L.codes_off = off;   off += 2u * (uint32_t)n * L.cw * 4u;
     L.scale_off = off;   off += 2u * (uint32_t)n * 4u;
     L.table_off = off;   off += (has_lut && code_bits <= 4) ? 2u * (uint32_t)n * 16u * 4u : 0u;
@@ -105,17 +105,18 @@ __device__ __forceinline__ void wide_column(const StepParams& p, const WideSmemL
             }
         }
         float s;
+        // two sets of partials, alternating: a fast warp may already write the
+        // next batch's partial while a slow one still reads this batch's
+        double* const red = reinterpret_cast<double*>(smem + L.red_off) + red_parity * (3 * npb * G);
+        if (G > 1 && !p.prescaled) red_parity ^= 1;
         if (p.prescaled) {
-            s = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+            if constexpr (T::kNorm) s = node_ok ? p.gmax[node] : 0.0f;       // the maximum that spans the grid
+            else s = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
         } else {
             double part;
             if constexpr (T::kSign) part = warp_sum(sum);
             else part = (double)__uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
             if (G > 1) {
-                // two sets of partials, alternating: a fast warp may already write the
-                // next batch's partial while a slow one still reads this batch's
-                double* red = reinterpret_cast<double*>(smem + L.red_off) + red_parity * (npb * G);
-                red_parity ^= 1;
                 if (lane == 0) red[grp * G + wg] = part;
                 __syncthreads();
                 part = 0.0;
@@ -136,6 +137,34 @@ __device__ __forceinline__ void wide_column(const StepParams& p, const WideSmemL
         const bool fast = T::kLut && s >= 0x1p-60f && s <= 0x1p+60f;
         const float inv_s = fast ? __fdiv_rn(1.0f, s) : 0.0f;
         const size_t code_row = (size_t)node * (size_t)p.code_pitch + (size_t)((k0 * T::kBits) >> 5);
+        // norm-matched codes: the whole chunk is coded first; s becomes the norm that is sent,
+        // dscale the factor the receiver applies to the levels
+        uint32_t qn[T::kNorm ? E : 1];
+        float cvn[T::kNorm ? E : 1];
+        float dscale = s;
+        if constexpr (T::kNorm) {
+            auto valid = [&](int t) { return node_ok && 4 * (f0 + fstride * (t >> 2)) + (t & 3) < m_len; };
+            double sv2, sl2;
+            norm_codes<CODE, E, FULL>(v, valid, s, lut, qn, cvn, sv2, sl2);
+            float nrm;
+            if (p.prescaled) {
+                nrm = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+                dscale = node_ok ? p.dscales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+            } else {
+                if (G > 1) {
+                    double* red2 = red + npb * G;
+                    double* red3 = red2 + npb * G;
+                    if (lane == 0) { red2[grp * G + wg] = sv2; red3[grp * G + wg] = sl2; }
+                    __syncthreads();
+                    sv2 = 0.0; sl2 = 0.0;
+                    for (int w = 0; w < G; ++w) { sv2 += red2[grp * G + w]; sl2 += red3[grp * G + w]; }
+                }
+                norm_finish(s, sv2, sl2, nrm, dscale);
+            }
+#pragma unroll
+            for (int t = 0; t < E; ++t) cvn[t] = __fmul_rn(dscale, cvn[t]);
+            s = nrm;
+        }
 #pragma unroll
         for (int r = 0; r < V; ++r) {
             const int f = f0 + fstride * r;
@@ -144,7 +173,13 @@ __device__ __forceinline__ void wide_column(const StepParams& p, const WideSmemL
             uint32_t piece = 0u;
             if (nv > 0) {
                 float cv[4];
-                if constexpr (T::kSign) {
+                if constexpr (T::kNorm) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        cv[j] = cvn[4 * r + j];
+                        if (FULL || j < nv) piece |= qn[4 * r + j] << (T::kBits * j);
+                    }
+                } else if constexpr (T::kSign) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         const uint32_t bit = (v[4 * r + j] >= 0.0f) ? 1u : 0u;
@@ -185,11 +220,14 @@ __device__ __forceinline__ void wide_column(const StepParams& p, const WideSmemL
         }
         if (node_ok && wg == 0) {
             if (lane == 0) {
-                scale_sm[node] = s;
-                if (!p.prescaled) p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+                scale_sm[node] = dscale_of<T::kNorm>(s, dscale);
+                if (!p.prescaled) {
+                    p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+                    if constexpr (T::kNorm) p.dscales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = dscale;
+                }
             }
             if constexpr (T::kTable) {
-                if (lane < (1 << T::kBits)) table_sm[node * 16 + lane] = __fmul_rn(s, lut[lane]);
+                if (lane < (1 << T::kBits)) table_sm[node * 16 + lane] = __fmul_rn(dscale_of<T::kNorm>(s, dscale), lut[lane]);
             }
         }
     }
@@ -270,6 +308,10 @@ __global__ void __launch_bounds__(512, 2) ds_wide_fused_kernel(const __grid_cons
     if constexpr (T::kLut) {
         float* lut = reinterpret_cast<float*>(smem + L.lut_off);
         for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x) lut[t] = p.lut[t];
+        // norm-matched codes: squares of the levels in binary64 (exact), in the unused part of the table
+        if constexpr (T::kNorm)
+            for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x)
+                reinterpret_cast<double*>(lut + 32)[t] = (double)p.lut[t] * (double)p.lut[t];
     }
     int32_t* rp = reinterpret_cast<int32_t*>(smem + L.rowptr_off);
     int32_t* cj = reinterpret_cast<int32_t*>(smem + L.col_off);

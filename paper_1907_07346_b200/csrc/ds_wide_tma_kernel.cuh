@@ -43,7 +43,7 @@ __host__ __device__ inline WideTmaSmemLayout wide_tma_smem_layout(int code_bits,
     L.scale_off = off;   off += 2u * (uint32_t)n * 4u;
     L.table_off = off;   off += (has_lut && code_bits <= 4) ? 2u * (uint32_t)n * 16u * 4u : 0u;
     off = (off + 7u) & ~7u;
-    L.red_off = off;     off += 2u * (uint32_t)nwarps * 8u;
+    L.red_off = off;     off += 2u * 3u * (uint32_t)nwarps * 8u;     // two alternating sets of (scale partial, two norm sums)
     L.mbar_off = off;    off += (uint32_t)nwarps * 8u;
     L.lut_off = off;     off += has_lut ? 256u * 4u : 0u;
     L.rowptr_off = off;  off += (uint32_t)(n + 1) * 4u;
@@ -57,7 +57,7 @@ __host__ __device__ inline WideTmaSmemLayout wide_tma_smem_layout(int code_bits,
 template <int CODE, int NOISE, int E>
 __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_constant__ StepParams p) {
     using T = CodeTraits<CODE>;
-    static_assert(!T::kIdentity && !T::kNorm, "identity and norm-matched codes run on other kernels");
+    static_assert(!T::kIdentity, "the identity compressor runs on other kernels");
     constexpr int V = E / 4;
     constexpr int SEG = E * 32;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -84,6 +84,10 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
 
     if constexpr (T::kLut)
         for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x) lut[t] = p.lut[t];
+    // norm-matched codes: squares of the levels in binary64 (exact), in the unused part of the table
+    if constexpr (T::kNorm)
+        for (int t = threadIdx.x; t < (1 << T::kBits); t += blockDim.x)
+            reinterpret_cast<double*>(lut + 32)[t] = (double)p.lut[t] * (double)p.lut[t];
     for (int t = threadIdx.x; t <= p.n; t += blockDim.x) rp[t] = p.row_ptr[t];
     for (int t = threadIdx.x; t < p.nnz; t += blockDim.x) { cj[t] = p.col_idx[t]; wp[t] = p.wprime[t]; }
     if (threadIdx.x < 2) abort_sm[threadIdx.x] = 0;
@@ -116,7 +120,7 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
     };
     // noise and rounding uniforms of item (col, b), Philox blocks in lockstep
     constexpr bool kGaussAhead = (NOISE == NOISE_GAUSS || NOISE == NOISE_T3);
-    constexpr bool kRndAhead = T::kLut;
+    constexpr bool kRndAhead = T::kLut && !T::kNorm;
     float zn[kGaussAhead ? E : 1];
     float mn[kRndAhead ? E : 1];
     auto draw = [&](int64_t col, int b) {
@@ -234,15 +238,16 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
 
                 // ---- scale ----
                 float s;
+                double* const red = reinterpret_cast<double*>(smem + L.red_off) + red_parity * (3 * nwarps);
+                if (G > 1 && !p.prescaled) red_parity ^= 1;
                 if (p.prescaled) {
-                    s = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+                    if constexpr (T::kNorm) s = node_ok ? p.gmax[node] : 0.0f;       // the maximum that spans the grid
+                    else s = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
                 } else {
                     double part;
                     if constexpr (T::kSign) part = warp_sum(sum);
                     else part = (double)__uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mx)));
                     if (G > 1) {
-                        double* red = reinterpret_cast<double*>(smem + L.red_off) + red_parity * nwarps;
-                        red_parity ^= 1;
                         if (lane == 0) red[warp] = part;
                         // only the G warps of this node meet (named barrier 1 + group): the other
                         // groups of the block are not held back
@@ -267,6 +272,34 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                 uint32_t* const codes_lane = p.codes + (size_t)(node_ok ? node : 0) * (size_t)p.code_pitch +
                                              (size_t)(((k0 + seg0) * T::kBits) >> 5) + lane / T::kLanesPerWord;
                 uint32_t* const codes_sm_lane = codes_sm + (size_t)(node_ok ? node : 0) * L.cw + word0 + lane / T::kLanesPerWord;
+                // norm-matched codes: the whole chunk is coded first; s becomes the norm that is
+                // sent, dscale the factor the receiver applies to the levels
+                uint32_t qn[T::kNorm ? E : 1];
+                float cvn[T::kNorm ? E : 1];
+                float dscale = s;
+                if constexpr (T::kNorm) {
+                    auto valid = [&](int t) { return 4 * (32 * (t >> 2) + lane) + (t & 3) < live_len; };
+                    double sv2, sl2;
+                    norm_codes<CODE, E, FULL>(v, valid, s, lut, qn, cvn, sv2, sl2);
+                    float nrm;
+                    if (p.prescaled) {
+                        nrm = node_ok ? p.scales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+                        dscale = node_ok ? p.dscales[(size_t)node * (size_t)p.scales_pitch] : 0.0f;
+                    } else {
+                        if (G > 1) {
+                            double* red2 = red + nwarps;
+                            double* red3 = red2 + nwarps;
+                            if (lane == 0) { red2[warp] = sv2; red3[warp] = sl2; }
+                            asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(32 * G) : "memory");
+                            sv2 = 0.0; sl2 = 0.0;
+                            for (int w = 0; w < G; ++w) { sv2 += red2[grp * G + w]; sl2 += red3[grp * G + w]; }
+                        }
+                        norm_finish(s, sv2, sl2, nrm, dscale);
+                    }
+#pragma unroll
+                    for (int t = 0; t < E; ++t) cvn[t] = __fmul_rn(dscale, cvn[t]);
+                    s = nrm;
+                }
 
                 // ---- phase B: compress, residual, pack ----
 #pragma unroll
@@ -276,7 +309,13 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                     uint32_t piece = 0u;
                     if (nv > 0) {
                         float cv[4];
-                        if constexpr (T::kSign) {
+                        if constexpr (T::kNorm) {
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                cv[j] = cvn[4 * r + j];
+                                if (FULL || j < nv) piece |= qn[4 * r + j] << (T::kBits * j);
+                            }
+                        } else if constexpr (T::kSign) {
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
                                 const uint32_t bit = (v[4 * r + j] >= 0.0f) ? 1u : 0u;
@@ -315,11 +354,14 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                 }
                 if (node_ok && alive && wg == 0) {
                     if (lane == 0) {
-                        scale_sm[node] = s;
-                        if (!p.prescaled) p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+                        scale_sm[node] = dscale_of<T::kNorm>(s, dscale);
+                        if (!p.prescaled) {
+                            p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+                            if constexpr (T::kNorm) p.dscales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = dscale;
+                        }
                     }
                     if constexpr (T::kTable) {
-                        if (lane < (1 << T::kBits)) table_sm[node * 16 + lane] = __fmul_rn(s, lut[lane]);
+                        if (lane < (1 << T::kBits)) table_sm[node * 16 + lane] = __fmul_rn(dscale_of<T::kNorm>(s, dscale), lut[lane]);
                     }
                 }
                 // the randomness of the next item, while its copies are in flight

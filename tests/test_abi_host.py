@@ -90,9 +90,8 @@ def test_init_argument_errors():
     assert _init(g, kind=B.DS_COMP_UNIFORM_STOCH_MAXABS, bits=3) == B.DS_ERR_UNSUPPORTED
     assert _init(g, kind=B.DS_COMP_SIGN1_L1, bits=2) == B.DS_ERR_UNSUPPORTED
     assert _init(g, chunk=32768) == B.DS_ERR_UNSUPPORTED
-    assert _init(g, kind=B.DS_COMP_UNIFORM_NEAREST_L2, bits=4, chunk=1024) == B.DS_ERR_UNSUPPORTED
     assert _init(g, kind=B.DS_COMP_UNIFORM_NEAREST_L2, bits=8, chunk=512) == B.DS_ERR_UNSUPPORTED
-    assert _init(g, kind=B.DS_COMP_UNIFORM_NEAREST_L2, bits=4, chunk=0) == B.DS_ERR_UNSUPPORTED
+    assert _init(g, kind=B.DS_COMP_UNIFORM_NEAREST_L2, bits=1, chunk=0) == B.DS_ERR_UNSUPPORTED
     assert _init(g, ws_bytes=1024) == B.DS_ERR_WORKSPACE
     st, ctx = B.ds_init_raw(None, g.col_idx, g.w, 8, 1000, 1024, 1, 1, 64, FAKE_WS, BIG)
     assert st == B.DS_ERR_NULL
@@ -155,6 +154,10 @@ def test_valid_init_reaches_cuda():
     is the first CUDA call.  (With a GPU the fake workspace pointer fails too.)"""
     for g in (I.ring(16), I.torus(4, 8), I.exponential(64)):
         _expect_ok_or_no_device(_init(g, N=4096, ld=4096, chunk=512))
+    # the norm-matched codec takes long chunks and one norm per node
+    for chunk in (1024, 0):
+        _expect_ok_or_no_device(_init(I.ring(8), N=4096, ld=4096, kind=B.DS_COMP_UNIFORM_NEAREST_L2, bits=4,
+                                      chunk=chunk))
 
 
 def test_null_handles():

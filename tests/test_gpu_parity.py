@@ -205,7 +205,8 @@ def test_single_step_other_noise(env, path, noise):
 
 
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("comp", [(I.COMP_SIGN1_L1, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 4)])
+@pytest.mark.parametrize("comp", [(I.COMP_SIGN1_L1, 1), (I.COMP_UNIFORM_STOCH_MAXABS, 4),
+                                  (I.COMP_UNIFORM_NEAREST_L2, 4), (I.COMP_UNIFORM_NEAREST_L2, 2)])
 @pytest.mark.parametrize("N", [65_536, 1000, 515])
 def test_per_node_scale(env, path, comp, N):
     run_case(env, I.ring(4), N, comp[0], comp[1], 0, I.NOISE_GAUSS, path)
@@ -411,6 +412,31 @@ def test_norm_matched_compressor_free_running(env, path, bits):
              steps=20, zero_start=True, tol=TOL_RUN, gamma=0.01)
     run_case(env, I.torus(4, 8), 256 * 5 + 7, I.COMP_UNIFORM_NEAREST_L2, bits, 256, I.NOISE_STUDENT_T3, path,
              steps=3)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("bits", [2, 4])
+def test_one_norm_per_tensor_free_running(env, path, bits):
+    """Section 5, "Compression" at the paper's granularity: b bits per element and ONE
+    Euclidean norm per tensor (chunk = 0: the node's whole vector), on the paper's topology
+    (8 workers on a ring), 20 free-running steps from zero; then many nodes (batches of nodes
+    per block), Student-t noise and a caller-tuned lane shape (several warps per tile)."""
+    torch, orc, B = env
+    run_case(env, I.ring(8), 512 * 37 + 41, I.COMP_UNIFORM_NEAREST_L2, bits, 0, I.NOISE_GAUSS, path,
+             steps=20, zero_start=True, tol=TOL_RUN, gamma=0.01)
+    run_case(env, I.exponential(64), 512 * 3 + 7, I.COMP_UNIFORM_NEAREST_L2, bits, 0, I.NOISE_STUDENT_T3, path,
+             steps=2)
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("chunk,graph", [(1024, I.ring(8)), (2048, I.ring(4)), (4096, I.ring(8)),
+                                         (1024, I.exponential(64)), (8192, I.ring(3))],
+                         ids=["1024x8", "2048x4", "4096x8", "1024x64", "8192x3"])
+def test_norm_matched_long_chunks(env, path, chunk, graph):
+    """Norm-matched codes on chunks that several warps share (the two sums of squares are
+    combined across the chunk's warps in warp order)."""
+    run_case(env, graph, chunk * 2 + chunk // 2 + 13, I.COMP_UNIFORM_NEAREST_L2, 4, chunk, I.NOISE_GAUSS, path,
+             steps=2)
 
 
 def test_compressed_runs_track_the_uncompressed_baseline(env):

@@ -335,3 +335,35 @@ def test_given_gradient_reproduces_synthetic_step(comp):
     assert np.allclose(v, H + d0, atol=2e-6, rtol=0)
     assert np.abs(Cv.astype(np.float64) + d3 - v).max() <= 2.4e-7 * max(1.0, np.abs(v).max())
     assert np.allclose(x3.astype(np.float64).mean(0), H.mean(0), atol=3e-6, rtol=0)
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_one_norm_per_tensor(bits):
+    """Section 5, "Compression": b bits per element and ONE Euclidean norm per
+    tensor, to which the receiver rescales what it decodes.  With chunk = 0
+    the whole row of a node is the tensor: the scalar sent is ||v_i||_2
+    (recomputed here in binary64 from v), the decoded C_i has that norm, the
+    codes are the nearest of the 2^b levels spanning [-max|v_i|, max|v_i|], and
+    C_i is a positive multiple of the decoded levels."""
+    g = I.ring(8)
+    N = 1000
+    x, d, a, c = make_problem(g, N, 5)
+    codes, scales, v, Cv = orc.step(g, I.COMP_UNIFORM_NEAREST_L2, bits, 0, x, d, a, c, N, 0.1,
+                                    I.NOISE_GAUSS, 0.05, 0.5, 9, 2, want_vC=True)
+    assert scales.shape == (8, 1)
+    L = (1 << bits) - 1
+    for i in range(8):
+        v64 = v[i].astype(np.float64)
+        assert abs(scales[i, 0] - np.sqrt((v64 ** 2).sum())) <= 1e-6 * scales[i, 0]
+        assert abs(np.sqrt((Cv[i].astype(np.float64) ** 2).sum()) - scales[i, 0]) <= 2e-6 * scales[i, 0]
+        q = np.zeros(N, np.int64)
+        for k in range(N):
+            q[k] = (int(codes[i, (k * bits) // 32]) >> ((k * bits) % 32)) & L
+        gmax = np.abs(v64).max()
+        levels = (2.0 * q - L) / L
+        # nearest level: no other level is closer to v / max|v| (up to the rounding of the quotient)
+        grid = (2.0 * np.arange(L + 1) - L) / L
+        best = np.abs(v64[:, None] / gmax - grid[None, :]).min(axis=1)
+        assert np.all(np.abs(v64 / gmax - levels) <= best + 1e-6)
+        ratio = Cv[i].astype(np.float64) / levels
+        assert np.all(ratio > 0) and np.ptp(ratio) <= 1e-6 * ratio.mean()
