@@ -12,7 +12,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdeepsqueeze.so")
+# DEEPSQUEEZE_LIB: load another build of the library (e.g. a checked or experimental one)
+LIB_PATH = os.environ.get("DEEPSQUEEZE_LIB") or os.path.join(_HERE, "libdeepsqueeze.so")
 
 DS_OK = 0
 (DS_ERR_NULL, DS_ERR_ARG, DS_ERR_GRAPH, DS_ERR_W_NOT_SYMMETRIC, DS_ERR_W_NOT_STOCHASTIC,

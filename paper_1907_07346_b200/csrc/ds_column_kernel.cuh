@@ -106,19 +106,32 @@ __device__ __forceinline__ void norm_codes(const float* v, ValidFn valid, float 
     // level[q]^2 in binary64, stored behind the 16 levels of the table: a product of two binary32
     // numbers is exact in binary64, so adding the stored square rounds exactly like the fused form
     const double* lut_sq = reinterpret_cast<const double*>(lut + 32);
+    // u + 1/2 for all elements: on the packed binary32x2 pipe when the reciprocal form of the
+    // quotient applies (each half rounds like the scalar operation), else element by element
+    float up[E];
+    if (fast) {
+        const float2 iv = splat(inv), hl = splat(kHalfL);
+#pragma unroll
+        for (int t = 0; t < E; t += 2) {
+            const float2 vv = make_float2(v[t], v[t + 1]);
+            const float2 q0 = __fmul2_rn(vv, iv);
+            const float2 rem = __ffma2_rn(make_float2(-q0.x, -q0.y), splat(m), vv);
+            const float2 y = __ffma2_rn(rem, iv, q0);
+            const float2 u = __ffma2_rn(y, hl, hl);
+            const float2 h = __fadd2_rn(u, splat(0.5f));
+            up[t] = h.x; up[t + 1] = h.y;
+        }
+    } else {
+#pragma unroll
+        for (int t = 0; t < E; ++t) {
+            const float y = dead ? 0.0f : __fdiv_rn(v[t], m);
+            up[t] = __fadd_rn(__fmaf_rn(y, kHalfL, kHalfL), 0.5f);
+        }
+    }
 #pragma unroll
     for (int t = 0; t < E; ++t) {
         const bool ok = FULL || valid(t);
-        float y;
-        if (fast) {
-            const float q0 = __fmul_rn(v[t], inv);
-            const float rem = __fmaf_rn(-q0, m, v[t]);
-            y = __fmaf_rn(rem, inv, q0);
-        } else {
-            y = dead ? 0.0f : __fdiv_rn(v[t], m);
-        }
-        const float u = __fmaf_rn(y, kHalfL, kHalfL);
-        const uint32_t code = dead ? 0u : (uint32_t)min(max(__float2int_rd(__fadd_rn(u, 0.5f)), 0), kLi);
+        const uint32_t code = dead ? 0u : (uint32_t)min(max(__float2int_rd(up[t]), 0), kLi);
         q[t] = code;
         lv[t] = lut[code];
         if (ok) {

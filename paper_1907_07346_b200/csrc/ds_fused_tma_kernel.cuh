@@ -107,6 +107,34 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+// L2 eviction policies and accesses that carry one.  Inputs that are read exactly once are
+// fetched "evict first", so that they do not push out lines that the same kernel re-reads.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar,
+                                              uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void st4_hint(float* p, float4 v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
+                 ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(policy) : "memory");
+}
+__device__ __forceinline__ float4 ld4_hint(const float* p, uint64_t policy) {
+    float4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(policy) : "memory");
+    return v;
+}
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -191,16 +219,13 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     // the rounding uniforms of the stochastic quantiser are drawn with it
     constexpr bool kRndAhead = T::kLut && !T::kNorm;
     float mn[kRndAhead ? E : 1];
-    // do_noise / do_rnd select which of the two streams are drawn by this call
-    auto draw_noise = [&](int64_t c, auto noise_tag, auto rnd_tag) {
-        constexpr bool DO_NOISE = decltype(noise_tag)::value && kNoiseAhead;
-        constexpr bool DO_RND = decltype(rnd_tag)::value && kRndAhead;
+    auto draw_noise = [&](int64_t c) {
         const uint32_t kbase = (uint32_t)(c * p.tile + seg0) + 4u * (uint32_t)lane;   // element of r = 0
-        if constexpr (DO_NOISE || DO_RND) {
-            // all Philox blocks of the call (V for the noise, V for the rounding stream,
-            // whichever are drawn) advance together
-            constexpr int kGauss = DO_NOISE ? V : 0;
-            constexpr int kRnd = DO_RND ? V : 0;
+        if constexpr (kNoiseAhead || kRndAhead) {
+            // all Philox blocks of the tile (V for the noise, V for the rounding stream,
+            // whichever are needed) advance together
+            constexpr int kGauss = kNoiseAhead ? V : 0;
+            constexpr int kRnd = kRndAhead ? V : 0;
             uint32_t stream[kGauss + kRnd], block[kGauss + kRnd];
             uint4 w[kGauss + kRnd];
 #pragma unroll
@@ -223,7 +248,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             }
         }
     };
-    if (col < p.tile_end) draw_noise(col, std::true_type{}, std::true_type{});      // (also when only the rounding stream is needed)
+    if (col < p.tile_end) draw_noise(col);      // (also when only the rounding stream is needed)
     uint32_t parity = 0;
     int buf = 0;
     uint32_t iter = 0;          // tiles this block has worked on
@@ -453,11 +478,6 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
             // before it is written again two tiles later.)
             __syncwarp();
             if (lane == 0) mbar_arrive(nbar0 + 8u * (uint32_t)(buf * p.n + node));
-            // The gradient noise of the next tile needs nothing from the neighbours: it is drawn
-            // HERE, between the announcement and the wait, so that by the time this warp looks at
-            // its neighbours' barriers they have normally completed and it does not poll.
-            const bool more = col + gridDim.x < p.tile_end;
-            if (more) draw_noise(col + gridDim.x, std::true_type{}, std::false_type{});
             {
                 const uint32_t nphase = (iter >> 1) & 1u;
                 bool ok = true;
@@ -504,8 +524,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                     st_partial(x_lane + 128 * r, make_float4(xa.x, xa.y, xb.x, xb.y), nv);
                 }
             }
-            // (the rounding uniforms of the next tile after the mix, when fewer registers are live)
-            if (more) draw_noise(col + gridDim.x, std::false_type{}, std::true_type{});
+            if (col + gridDim.x < p.tile_end) draw_noise(col + gridDim.x);
             return false;
         };
         const bool aborted = full ? tile_body(std::true_type{}) : tile_body(std::false_type{});

@@ -95,6 +95,13 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
+#ifndef DS_WIDE_L2_HINTS
+#define DS_WIDE_L2_HINTS 3
+#endif
+#if DS_WIDE_L2_HINTS
+    const uint64_t pol_first = l2_policy_evict_first();
+    const uint64_t pol_last = l2_policy_evict_last();
+#endif
     auto seg_len_of = [&](int64_t col) -> int {
         const int64_t remain = p.N - col * p.tile;
         const int m_len = (int)(remain < p.tile ? remain : p.tile);
@@ -111,10 +118,18 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
             fence_proxy_async();
             constexpr uint32_t kArrays = (NOISE == GRAD_GIVEN) ? 3u : 4u;
             mbar_expect_tx(bar, kArrays * bytes);
+#if DS_WIDE_L2_HINTS & 1
+            // read once: must not push the parked x - gamma g out of L2 before the second sweep
+            bulk_g2s_hint(slot_addr + 0u * L.seg_bytes, p.x + at, bytes, bar, pol_first);
+            bulk_g2s_hint(slot_addr + 1u * L.seg_bytes, p.delta + at, bytes, bar, pol_first);
+            bulk_g2s_hint(slot_addr + 2u * L.seg_bytes, p.a + at, bytes, bar, pol_first);
+            if constexpr (NOISE != GRAD_GIVEN) bulk_g2s_hint(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar, pol_first);
+#else
             bulk_g2s(slot_addr + 0u * L.seg_bytes, p.x + at, bytes, bar);
             bulk_g2s(slot_addr + 1u * L.seg_bytes, p.delta + at, bytes, bar);
             bulk_g2s(slot_addr + 2u * L.seg_bytes, p.a + at, bytes, bar);
             if constexpr (NOISE != GRAD_GIVEN) bulk_g2s(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar);
+#endif
         }
         return true;
     };
@@ -217,7 +232,12 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                             local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, h, &v[4 * r]);
                         }
                         if (FULL || nv == 4) {
+#if DS_WIDE_L2_HINTS & 2
+                            // parked for the second sweep: keep it in L2 until then
+                            st4_hint(x_lane + 128 * r, make_float4(h[0], h[1], h[2], h[3]), pol_last);
+#else
                             *reinterpret_cast<float4*>(x_lane + 128 * r) = make_float4(h[0], h[1], h[2], h[3]);
+#endif
                         } else {
                             for (int j = 0; j < nv; ++j) x_lane[128 * r + j] = h[j];
                         }
@@ -388,7 +408,11 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                     const int nv = FULL ? 4 : min(max(seg_len - e0, 0), 4);
                     hv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (nv == 4) {
+#if DS_WIDE_L2_HINTS & 2
+                        hv[r] = ld4_hint(x_lane + 128 * r, pol_first);      // last use of the parked line
+#else
                         hv[r] = *reinterpret_cast<const float4*>(x_lane + 128 * r);
+#endif
                     } else if (nv > 0) {
                         float* hp = reinterpret_cast<float*>(&hv[r]);
                         for (int j = 0; j < nv; ++j) hp[j] = x_lane[128 * r + j];
