@@ -56,7 +56,9 @@ typedef enum {
     DS_ERR_WORKSPACE = 8,        /* workspace smaller than ds_workspace_size() */
     DS_ERR_UNSUPPORTED = 9,      /* combination not implemented (e.g. bits not in {1,2,4,8}) */
     DS_ERR_CUDA = 10,            /* a CUDA runtime call failed (no device, launch error, ...) */
-    DS_ERR_TIMEOUT = 11          /* a bounded wait inside a kernel ran out; x, delta are incomplete */
+    DS_ERR_TIMEOUT = 11,         /* a bounded wait inside a kernel ran out; x, delta are incomplete */
+    DS_ERR_BOUNDS = 12           /* checked build only: a kernel computed an index outside its arrays; that
+                                    part of the step was skipped, nothing out of range was touched */
 } ds_status;
 
 /* Node graph in CSR form, HOST memory: row i lists N(i) in ascending order
@@ -332,6 +334,17 @@ ds_status ds_selftest_math(uint64_t *counts, void *cuda_stream);
  * not arrive.  The next ds_sync must return DS_ERR_TIMEOUT (and clear the flag).
  * Nothing hangs and nothing faults; x and delta are not touched. */
 ds_status ds_selftest_timeout(ds_ctx *ctx, void *cuda_stream);
+
+/* Checked build (the library compiled with -DDS_DEBUG, `python -m
+ * paper_1907_07346_b200.build --debug`): before a warp touches its part of a row,
+ * the kernels validate the indices behind every access of that part -- row,
+ * first element, length, code words, scale slot, partial slot -- against the
+ * shape; a part that fails is skipped and ds_sync returns DS_ERR_BOUNDS (once;
+ * nothing traps, nothing out of range is read or written).  The checked build
+ * computes the same results as the normal one.  This self-test asks the checker
+ * about a part in the row after the last one: the next ds_sync must return
+ * DS_ERR_BOUNDS.  In the normal build it returns DS_ERR_UNSUPPORTED. */
+ds_status ds_selftest_bounds(ds_ctx *ctx, void *cuda_stream);
 
 /* Diagnostics: write the random streams the kernels draw from, one value per
  * element, out[node][k] for k < N (device, [n][ld_out]).  which = 0: unit

@@ -18,7 +18,7 @@ LIB_PATH = os.environ.get("DEEPSQUEEZE_LIB") or os.path.join(_HERE, "libdeepsque
 DS_OK = 0
 (DS_ERR_NULL, DS_ERR_ARG, DS_ERR_GRAPH, DS_ERR_W_NOT_SYMMETRIC, DS_ERR_W_NOT_STOCHASTIC,
  DS_ERR_NO_SELF_LOOP, DS_ERR_ALIGN, DS_ERR_WORKSPACE, DS_ERR_UNSUPPORTED, DS_ERR_CUDA,
- DS_ERR_TIMEOUT) = range(1, 12)
+ DS_ERR_TIMEOUT, DS_ERR_BOUNDS) = range(1, 13)
 
 DS_COMP_IDENTITY, DS_COMP_SIGN1_L1, DS_COMP_UNIFORM_STOCH_MAXABS, DS_COMP_UNIFORM_NEAREST_L2 = 0, 1, 2, 3
 DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
@@ -27,7 +27,7 @@ DS_RUN_MAX_STEPS = 4096
 DS_RESIDENT_MAX_STEPS = 1024
 
 EXPORTS = ["ds_workspace_size", "ds_init", "ds_step", "ds_step_g", "ds_ecsgd_step", "ds_ecsgd_step_g", "ds_run", "ds_run_resident", "ds_step_host", "ds_codes", "ds_set_path",
-           "ds_tune", "ds_get_info", "ds_sync", "ds_selftest_timeout", "ds_selftest_math", "ds_noise", "ds_node_scales_noalloc",
+           "ds_tune", "ds_get_info", "ds_sync", "ds_selftest_timeout", "ds_selftest_bounds", "ds_selftest_math", "ds_noise", "ds_node_scales_noalloc",
            "ds_destroy", "ds_strerror"]
 
 
@@ -103,6 +103,8 @@ def lib():
         L.ds_sync.restype = C.c_int
         L.ds_selftest_timeout.argtypes = [C.c_void_p, C.c_void_p]
         L.ds_selftest_timeout.restype = C.c_int
+        L.ds_selftest_bounds.argtypes = [C.c_void_p, C.c_void_p]
+        L.ds_selftest_bounds.restype = C.c_int
         L.ds_selftest_math.argtypes = [C.c_void_p, C.c_void_p]
         L.ds_selftest_math.restype = C.c_int
         L.ds_noise.argtypes = [C.c_void_p, C.c_int32, C.c_int64, C.c_int64, C.c_int32, C.c_int32,
@@ -297,6 +299,11 @@ class DeepSqueeze:
     def ds_selftest_timeout(self, stream=None):
         s = self.torch.cuda.current_stream(self.device) if stream is None else stream
         _check(lib().ds_selftest_timeout(self.ctx, C.c_void_p(s.cuda_stream)), "ds_selftest_timeout")
+
+    def ds_selftest_bounds(self, stream=None) -> int:
+        """Returns the ds_status (DS_ERR_UNSUPPORTED unless the library is the checked build)."""
+        s = self.torch.cuda.current_stream(self.device) if stream is None else stream
+        return int(lib().ds_selftest_bounds(self.ctx, C.c_void_p(s.cuda_stream)))
 
     def ds_codes(self):
         """(codes_ptr, code_pitch_words, scales_ptr, scales_pitch) of the last step."""

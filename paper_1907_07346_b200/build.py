@@ -1,6 +1,6 @@
 """Build libdeepsqueeze.so (CUDA, sm_100a only) in-tree with nvcc.
 
-    python -m paper_1907_07346_b200.build [--force] [--verbose]
+    python -m paper_1907_07346_b200.build [--force] [--verbose] [--debug]
 
 -fmad=false: the kernels spell out every fused multiply-add themselves
 (__fmaf_rn); the compiler must not contract any other a*b+c, because packed
@@ -44,12 +44,27 @@ def _newest(paths) -> float:
     return max(os.path.getmtime(p) for p in list(paths) + [os.path.abspath(__file__)])
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
-    extra = ["-Xptxas", "-v"] if verbose else []
+LIB_DEBUG = os.path.join(HERE, "libdeepsqueeze_debug.so")
+OBJ_DEBUG = os.path.join(HERE, "_build_debug")
+
+
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """debug=True: the checked build (-DDS_DEBUG: the kernels validate their index
+    arithmetic and report instead of touching memory out of range) as
+    libdeepsqueeze_debug.so; load it with DEEPSQUEEZE_LIB=<that path>."""
+    obj_dir, lib = (OBJ_DEBUG, LIB_DEBUG) if debug else (OBJ, LIB)
+    extra = (["-Xptxas", "-v"] if verbose else []) + (["-DDS_DEBUG"] if debug else [])
+    if debug and not force and os.path.exists(lib):
+        # an up-to-date library is enough (its object files need not be kept)
+        sources = set()
+        for src in SOURCES:
+            _deps(os.path.join(CSRC, src), sources)
+        if os.path.getmtime(lib) >= _newest(sources):
+            return lib
+    os.makedirs(obj_dir, exist_ok=True)
 
     def compile_one(src: str) -> str:
-        obj = os.path.join(OBJ, src.replace(".cu", ".o"))
+        obj = os.path.join(obj_dir, src.replace(".cu", ".o"))
         path = os.path.join(CSRC, src)
         # an object is rebuilt when its source or anything it includes is newer
         if not force and os.path.exists(obj) and os.path.getmtime(obj) >= _newest(_deps(path)):
@@ -64,11 +79,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with ThreadPoolExecutor(max_workers=len(SOURCES)) as ex:
         objs = list(ex.map(compile_one, SOURCES))
-    if force or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
+    if force or not os.path.exists(lib) or os.path.getmtime(lib) < max(os.path.getmtime(o) for o in objs):
         subprocess.run(["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a",
-                        "-o", LIB, *objs], check=True)
-    return LIB
+                        "-o", lib, *objs], check=True)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

@@ -184,7 +184,7 @@ __device__ __forceinline__ void st_partial(float* p, float4 v, int nv) {
 template <int CODE, int NOISE, int E, int MODE, bool FULL>
 __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayout& L,
                                             unsigned char* smem, int64_t col, int buf,
-                                            int lane, int grp, int wg, int node, bool node_ok) {
+                                            int lane, int grp, int wg, int node, bool node_ok) {   // (node_ok: by value)
     using T = CodeTraits<CODE>;
     constexpr int V = E / 4;
     const int G = p.warps_per_group;
@@ -194,6 +194,13 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
     const int fstride = 32 * G;
     const int f0 = wg * 32 + lane;
     const size_t row = (size_t)node * (size_t)p.ld + (size_t)k0;
+    // checked build: a refused (node, tile) is treated like a node beyond the last one
+    // (no loads, no stores; the block's barriers are still met)
+    if (DS_CHECKED_BUILD && node_ok &&
+        !ds_part_ok(p, node, k0, m_len, MODE == MODE_REDUCE ? 0 : T::kBits,      // (a reduction writes no codes)
+                    (T::kIdentity || p.prescaled || MODE == MODE_REDUCE) ? -1 : col))
+        node_ok = false;
+    if (DS_CHECKED_BUILD && MODE == MODE_REDUCE && node_ok && !ds_partial_ok(p, node, p.n, col)) node_ok = false;
 
     float h[E], v[E];
 
@@ -416,6 +423,7 @@ __device__ __forceinline__ void column_body(const StepParams& p, const SmemLayou
             if (wg == 0 && lane < (1 << T::kBits)) table_sm[grp * 16 + lane] = __fmul_rn(dscale, lut[lane]);
         }
         __syncthreads();    // codes and scales of all nodes of this tile are in shared memory
+        if (!node_ok) return;
 
         // the tile's packed codes leave for global memory ("send")
         const int cw_valid = (m_len * T::kBits + 31) >> 5;

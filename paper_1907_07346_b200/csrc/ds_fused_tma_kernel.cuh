@@ -194,6 +194,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
     auto issue = [&](int64_t col) -> bool {
         const int len = seg_len_of(col);
         if (len <= 0) return false;
+        if (DS_CHECKED_BUILD && !ds_part_ok(p, node, col * p.tile + seg0, len, T::kBits, -1)) return false;
         if (lane == 0) {
             const uint32_t bytes = (uint32_t)((len + 3) & ~3) * 4u;
             const size_t at = (size_t)node * (size_t)p.ld + (size_t)(col * p.tile) + (size_t)seg0;
@@ -283,6 +284,11 @@ __global__ void __launch_bounds__(MAXT, 1) ds_fused_tma_kernel(const __grid_cons
                 abort_sm[buf] = 1;
                 if (lane == 0) *p.error_flag = 1;
             }
+        }
+        if (DS_CHECKED_BUILD && seg_len > 0 &&
+            !ds_part_ok(p, node, k0 + seg0, seg_len, T::kBits, (T::kIdentity || p.prescaled) ? -1 : col)) {
+            alive = false;              // refused: the warp stores nothing and the block winds down
+            abort_sm[buf] = 1;
         }
         const int live_len = alive ? seg_len : 0;
         const bool full = (live_len == SEG);

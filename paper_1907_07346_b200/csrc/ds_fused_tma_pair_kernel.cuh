@@ -161,6 +161,11 @@ __global__ void __launch_bounds__(512, 1) ds_fused_tma_pair_kernel(const __grid_
                 if (lane == 0) *p.error_flag = 1;
             }
         }
+        if (DS_CHECKED_BUILD &&
+            !(ds_part_ok(p, node_of[0], k0, m_len, T::kBits, col) && ds_part_ok(p, node_of[NPW - 1], k0, m_len, T::kBits, col))) {
+            alive = false;              // refused: the warp stores nothing and the block winds down
+            abort_sm[buf] = 1;
+        }
         const int live_len = alive ? m_len : 0;
         const bool full = (live_len == SUB);
 

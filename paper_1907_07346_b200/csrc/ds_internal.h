@@ -44,18 +44,67 @@ struct StepParams {
     double* partials;         // [n][tiles], per-node-scale reduction (twice that for the two sums of a
                               // per-node norm: sum v^2 in the first half, sum level^2 in the second)
     float* gmax;              // [n], norm-matched codes with one norm per node: max |v| of the node
-    int* error_flag;          // set to 1 by a kernel whose bounded wait ran out
+    int* error_flag;          // DS_FLAG_* bits: a bounded wait ran out; the checked build refused an index
     float sigma;
     float neg_gamma;
     float eta;
     RngStep rs;
     int32_t warps_per_group;  // warps sharing one (node, tile)
     int32_t nodes_per_block;
+    int32_t l2_hints;         // batch-sweeping TMA kernel: bit 0 = inputs evict-first, bit 1 = parked values evict-last
     int32_t prescaled;        // 1: scale of node i is scales[i][0], computed by an earlier launch
     int32_t norm_phase;       // reduce mode, norm-matched codes, one norm per node: 0 = maximum, 2 = sums of squares
     int32_t ecsgd;            // 1 (compress / reduce modes only): centralized error-compensated SGD,
                               // v = g + delta is compressed and x is left for the server's update
 };
+
+// Values of the error flag (bits): a bounded wait ran out / the checked build
+// refused an out-of-range index.
+enum : int { DS_FLAG_TIMEOUT = 1, DS_FLAG_BOUNDS = 2 };
+
+// Checked build (-DDS_DEBUG): before a warp touches its part of a row, the index
+// arithmetic behind every access of that part is validated here; a part that
+// does not lie inside the row, its code words and its scale slot is NOT
+// processed, and the error flag records it (ds_sync then returns
+// DS_ERR_BOUNDS).  Nothing traps.  In the normal build this is `true` and
+// the compiler removes the call.
+//   node       row
+//   k_first    first element of the part within the row
+//   count      elements of the part that are read and written (the staging
+//              copies read count rounded up to 4: padding columns up to ld)
+//   code_bits  bits per packed code
+//   scale_col  index of the scale the part writes within the row's scales, -1 = none
+#ifdef DS_DEBUG
+#define DS_CHECKED_BUILD 1
+#else
+#define DS_CHECKED_BUILD 0
+#endif
+__device__ __forceinline__ bool ds_part_ok(const StepParams& p, int64_t node, int64_t k_first, int64_t count,
+                                           int code_bits, int64_t scale_col) {
+#if DS_CHECKED_BUILD
+    bool ok = node >= 0 && node < p.n && k_first >= 0 && count >= 0;
+    ok = ok && (k_first & 3) == 0;                                   // 128-bit accesses
+    ok = ok && k_first + count <= p.N && k_first + ((count + 3) & ~(int64_t)3) <= p.ld;
+    ok = ok && (((k_first + count) * code_bits + 31) >> 5) <= p.code_pitch;
+    ok = ok && scale_col < p.scales_pitch;
+    if (!ok && p.error_flag != nullptr) atomicOr(p.error_flag, (int)DS_FLAG_BOUNDS);
+    return ok;
+#else
+    (void)p; (void)node; (void)k_first; (void)count; (void)code_bits; (void)scale_col;
+    return true;
+#endif
+}
+// The same for one slot of the per-(node, tile) partials (`rows` rows of p.tiles slots).
+__device__ __forceinline__ bool ds_partial_ok(const StepParams& p, int64_t row, int64_t rows, int64_t col) {
+#if DS_CHECKED_BUILD
+    const bool ok = row >= 0 && row < rows && col >= 0 && col < p.tiles;
+    if (!ok && p.error_flag != nullptr) atomicOr(p.error_flag, (int)DS_FLAG_BOUNDS);
+    return ok;
+#else
+    (void)p; (void)row; (void)rows; (void)col;
+    return true;
+#endif
+}
 
 struct LaunchShape {
     int code;                 // CODE_*
@@ -82,6 +131,7 @@ cudaError_t launch_finalize_norms(const StepParams& p, cudaStream_t stream);
 cudaError_t launch_mix_kernel(const StepParams& p, int code, cudaStream_t stream);
 cudaError_t launch_math_selftest(unsigned long long* counts, cudaStream_t stream);
 cudaError_t launch_wait_selftest(int* error_flag, cudaStream_t stream);
+cudaError_t launch_bounds_selftest(const StepParams& p, cudaStream_t stream);
 cudaError_t launch_noise_kernel(float* out, int32_t n, int64_t N, int64_t ld, int which, int noise,
                                 RngStep rs, cudaStream_t stream);
 

@@ -30,6 +30,7 @@ __global__ void __launch_bounds__(256) ds_mix_kernel(const __grid_constant__ Ste
         const int64_t k = 4 * f;
         const int nv = (int)min((int64_t)4, p.N - k);
         const int64_t tile_idx = p.prescaled ? 0 : k / p.tile;
+        if (DS_CHECKED_BUILD && !ds_part_ok(p, node, k, nv, T::kBits, T::kIdentity ? -1 : tile_idx)) continue;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         for (int e = e_beg; e < e_end; ++e) {
             const int j = p.col_idx[e];
@@ -101,6 +102,7 @@ __global__ void __launch_bounds__(32) ds_finalize_scales_kernel(const __grid_con
     const int node = blockIdx.x;
     const int lane = threadIdx.x;
     const double* part = p.partials + (size_t)node * (size_t)p.tiles;
+    if (DS_CHECKED_BUILD && !ds_partial_ok(p, node, p.n, p.tiles - 1)) return;
     double acc = 0.0;
     for (int64_t t = lane; t < p.tiles; t += 32) acc = sign ? acc + part[t] : fmax(acc, part[t]);
 #pragma unroll
@@ -140,6 +142,7 @@ __global__ void __launch_bounds__(32) ds_finalize_norms_kernel(const __grid_cons
     const int lane = threadIdx.x;
     const double* pv = p.partials + (size_t)node * (size_t)p.tiles;
     const double* pl = p.partials + ((size_t)p.n + (size_t)node) * (size_t)p.tiles;
+    if (DS_CHECKED_BUILD && !ds_partial_ok(p, (int64_t)p.n + node, 2 * (int64_t)p.n, p.tiles - 1)) return;
     double sv2 = 0.0, sl2 = 0.0;
     for (int64_t t = lane; t < p.tiles; t += 32) { sv2 += pv[t]; sl2 += pl[t]; }
 #pragma unroll
@@ -233,6 +236,17 @@ __global__ void __launch_bounds__(256) ds_math_selftest_kernel(unsigned long lon
 
 cudaError_t launch_math_selftest(unsigned long long* counts, cudaStream_t stream) {
     ds_math_selftest_kernel<<<148 * 8, 256, 0, stream>>>(counts);
+    return cudaGetLastError();
+}
+
+// Self-test of the checked build: asks the checker about a part that starts in the row
+// after the last one.  It must refuse it (and raise the flag); nothing is accessed.
+__global__ void __launch_bounds__(32) ds_bounds_selftest_kernel(const __grid_constant__ StepParams p) {
+    if (threadIdx.x == 0) (void)ds_part_ok(p, p.n, 0, 4, 1, -1);
+}
+
+cudaError_t launch_bounds_selftest(const StepParams& p, cudaStream_t stream) {
+    ds_bounds_selftest_kernel<<<1, 32, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

@@ -100,6 +100,7 @@ extern "C" ds_status ds_node_scales_noalloc(float* scales_out, const float* x, c
     p.scales = scales_out;
     p.dscales = scales_out;
     p.scales_pitch = 1;
+    p.code_pitch = (N * 4 + 31) / 32;       // no codes are written; what a row of 4-bit codes would take (checked build)
     p.sigma = gp->sigma;
     p.neg_gamma = -gamma;
     p.eta = 0.0f;

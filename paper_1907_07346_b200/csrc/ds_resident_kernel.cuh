@@ -78,7 +78,11 @@ __global__ void __launch_bounds__(MAXT, 1) ds_resident_kernel(const __grid_const
     const int64_t col = blockIdx.x;                     // one tile per block
     const int64_t k0 = col * SEG;
     const int64_t remain = p.N - k0;
-    const int m_len = (int)(remain < SEG ? remain : SEG);
+    int m_len = (int)(remain < SEG ? remain : SEG);
+    // checked build: a refused tile is worked on as an empty one (nothing loaded, nothing stored;
+    // the block still takes part in the grid barrier)
+    bool part_ok = true;
+    if (DS_CHECKED_BUILD && !ds_part_ok(p, node, k0, m_len, T::kBits, p.prescaled ? -1 : col)) { part_ok = false; m_len = 0; }
 
     float* ac = reinterpret_cast<float*>(smem + L.ac_off) + (size_t)node * 2 * SEG;
     float* cval = reinterpret_cast<float*>(smem + L.cval_off);
@@ -214,7 +218,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_resident_kernel(const __grid_const
         // one scale per node: publish the tile's partial and arrive at the grid barrier ...
         double* mine = rp.partials2 + (size_t)(t & 1) * (size_t)p.n * (size_t)p.tiles;
         if (p.prescaled) {
-            if (lane == 0) mine[(size_t)node * (size_t)p.tiles + (size_t)col] = part;
+            if (lane == 0 && part_ok) mine[(size_t)node * (size_t)p.tiles + (size_t)col] = part;
             __syncthreads();
             if (threadIdx.x == 0) {
                 __threadfence();
@@ -269,7 +273,7 @@ __global__ void __launch_bounds__(MAXT, 1) ds_resident_kernel(const __grid_const
                 s = (float)part;
                 if (s == 0.0f || !(fabsf(s) <= 3.402823466e+38f)) s = 0.0f;
             }
-            if (lane == 0) p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
+            if (lane == 0 && part_ok) p.scales[(size_t)node * (size_t)p.scales_pitch + (size_t)col] = s;
         }
 
         // ---- compress, residual, pack; C[v] to shared memory ----

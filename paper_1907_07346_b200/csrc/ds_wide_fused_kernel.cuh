@@ -66,7 +66,9 @@ __device__ __forceinline__ void wide_column(const StepParams& p, const WideSmemL
     // ---------------- sweep 1: compress every batch of nodes ----------------
     for (int b = 0; b < batches; ++b) {
         const int node = b * npb + grp;
-        const bool node_ok = node < p.n;
+        bool node_ok = node < p.n;
+        // checked build: a refused (node, tile) is treated like a node beyond the last one
+        if (DS_CHECKED_BUILD && node_ok && !ds_part_ok(p, node, k0, m_len, T::kBits, p.prescaled ? -1 : col)) node_ok = false;
         const size_t row = (size_t)node * (size_t)p.ld + (size_t)k0;
         float v[E];
         double sum = 0.0;
@@ -240,6 +242,7 @@ __device__ __forceinline__ void wide_column(const StepParams& p, const WideSmemL
     for (int b = 0; b < batches; ++b) {
         const int node = b * npb + grp;
         if (node >= p.n) continue;
+        if (DS_CHECKED_BUILD && !ds_part_ok(p, node, k0, m_len, T::kBits, -1)) continue;
         const size_t row = (size_t)node * (size_t)p.ld + (size_t)k0;
         float acc[E];
 #pragma unroll

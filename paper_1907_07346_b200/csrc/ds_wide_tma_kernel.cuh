@@ -95,13 +95,14 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
-#ifndef DS_WIDE_L2_HINTS
-#define DS_WIDE_L2_HINTS 3
-#endif
-#if DS_WIDE_L2_HINTS
+    // L2 eviction hints, chosen by the host from the shape (StepParams::l2_hints):
+    //   bit 0  the staged inputs are fetched "evict first" (read once; with many nodes per column
+    //          they would otherwise push the parked x - gamma g out of L2 before the second sweep)
+    //   bit 1  x - gamma g is parked "evict last" and re-read "evict first"
     const uint64_t pol_first = l2_policy_evict_first();
     const uint64_t pol_last = l2_policy_evict_last();
-#endif
+    const bool hint_inputs = (p.l2_hints & 1) != 0;
+    const bool hint_parked = (p.l2_hints & 2) != 0;
     auto seg_len_of = [&](int64_t col) -> int {
         const int64_t remain = p.N - col * p.tile;
         const int m_len = (int)(remain < p.tile ? remain : p.tile);
@@ -112,24 +113,24 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
         const int node = b * npb + grp;
         const int len = seg_len_of(col);
         if (node >= p.n || len <= 0) return false;
+        if (DS_CHECKED_BUILD && !ds_part_ok(p, node, col * p.tile + seg0, len, T::kBits, -1)) return false;
         if (lane == 0) {
             const uint32_t bytes = (uint32_t)((len + 3) & ~3) * 4u;
             const size_t at = (size_t)node * (size_t)p.ld + (size_t)(col * p.tile) + (size_t)seg0;
             fence_proxy_async();
             constexpr uint32_t kArrays = (NOISE == GRAD_GIVEN) ? 3u : 4u;
             mbar_expect_tx(bar, kArrays * bytes);
-#if DS_WIDE_L2_HINTS & 1
-            // read once: must not push the parked x - gamma g out of L2 before the second sweep
-            bulk_g2s_hint(slot_addr + 0u * L.seg_bytes, p.x + at, bytes, bar, pol_first);
-            bulk_g2s_hint(slot_addr + 1u * L.seg_bytes, p.delta + at, bytes, bar, pol_first);
-            bulk_g2s_hint(slot_addr + 2u * L.seg_bytes, p.a + at, bytes, bar, pol_first);
-            if constexpr (NOISE != GRAD_GIVEN) bulk_g2s_hint(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar, pol_first);
-#else
-            bulk_g2s(slot_addr + 0u * L.seg_bytes, p.x + at, bytes, bar);
-            bulk_g2s(slot_addr + 1u * L.seg_bytes, p.delta + at, bytes, bar);
-            bulk_g2s(slot_addr + 2u * L.seg_bytes, p.a + at, bytes, bar);
-            if constexpr (NOISE != GRAD_GIVEN) bulk_g2s(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar);
-#endif
+            if (hint_inputs) {
+                bulk_g2s_hint(slot_addr + 0u * L.seg_bytes, p.x + at, bytes, bar, pol_first);
+                bulk_g2s_hint(slot_addr + 1u * L.seg_bytes, p.delta + at, bytes, bar, pol_first);
+                bulk_g2s_hint(slot_addr + 2u * L.seg_bytes, p.a + at, bytes, bar, pol_first);
+                if constexpr (NOISE != GRAD_GIVEN) bulk_g2s_hint(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar, pol_first);
+            } else {
+                bulk_g2s(slot_addr + 0u * L.seg_bytes, p.x + at, bytes, bar);
+                bulk_g2s(slot_addr + 1u * L.seg_bytes, p.delta + at, bytes, bar);
+                bulk_g2s(slot_addr + 2u * L.seg_bytes, p.a + at, bytes, bar);
+                if constexpr (NOISE != GRAD_GIVEN) bulk_g2s(slot_addr + 3u * L.seg_bytes, p.c + at, bytes, bar);
+            }
         }
         return true;
     };
@@ -198,6 +199,11 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                     if (lane == 0) *p.error_flag = 1;
                 }
             }
+            if (DS_CHECKED_BUILD && node_ok && seg_len > 0 &&
+                !ds_part_ok(p, node, k0 + seg0, seg_len, T::kBits, p.prescaled ? -1 : col)) {
+                alive = false;          // refused: the warp stores nothing and the block stops after this sweep
+                abort_sm[buf] = 1;
+            }
             const int live_len = (alive && node_ok) ? seg_len : 0;
             const bool full = (live_len == SEG);
             const int nb = (b + 1 < batches) ? b + 1 : 0;
@@ -232,12 +238,9 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                             local_step4(x4, d4, a4, c4, z4, p.sigma, p.neg_gamma, h, &v[4 * r]);
                         }
                         if (FULL || nv == 4) {
-#if DS_WIDE_L2_HINTS & 2
-                            // parked for the second sweep: keep it in L2 until then
-                            st4_hint(x_lane + 128 * r, make_float4(h[0], h[1], h[2], h[3]), pol_last);
-#else
-                            *reinterpret_cast<float4*>(x_lane + 128 * r) = make_float4(h[0], h[1], h[2], h[3]);
-#endif
+                            // parked for the second sweep
+                            if (hint_parked) st4_hint(x_lane + 128 * r, make_float4(h[0], h[1], h[2], h[3]), pol_last);
+                            else *reinterpret_cast<float4*>(x_lane + 128 * r) = make_float4(h[0], h[1], h[2], h[3]);
                         } else {
                             for (int j = 0; j < nv; ++j) x_lane[128 * r + j] = h[j];
                         }
@@ -397,6 +400,7 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
         for (int b = 0; b < batches; ++b) {
             const int node = b * npb + grp;
             if (node >= p.n || seg_len <= 0) continue;
+            if (DS_CHECKED_BUILD && !ds_part_ok(p, node, k0 + seg0, seg_len, T::kBits, -1)) continue;
             float* const x_lane = p.x + (size_t)node * (size_t)p.ld + (size_t)k0 + (size_t)seg0 + 4 * lane;
             auto mix_body = [&](auto full_tag) {
                 constexpr bool FULL = decltype(full_tag)::value;
@@ -408,11 +412,8 @@ __global__ void __launch_bounds__(512, 1) ds_wide_tma_kernel(const __grid_consta
                     const int nv = FULL ? 4 : min(max(seg_len - e0, 0), 4);
                     hv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (nv == 4) {
-#if DS_WIDE_L2_HINTS & 2
-                        hv[r] = ld4_hint(x_lane + 128 * r, pol_first);      // last use of the parked line
-#else
-                        hv[r] = *reinterpret_cast<const float4*>(x_lane + 128 * r);
-#endif
+                        if (hint_parked) hv[r] = ld4_hint(x_lane + 128 * r, pol_first);      // last use of the parked line
+                        else hv[r] = *reinterpret_cast<const float4*>(x_lane + 128 * r);
                     } else if (nv > 0) {
                         float* hp = reinterpret_cast<float*>(&hv[r]);
                         for (int j = 0; j < nv; ++j) hp[j] = x_lane[128 * r + j];
