@@ -251,7 +251,7 @@ def other_workload_line(torch, B, name: str, steps: int, dev, local_rank: int, p
     achieved = b_alg * w.n * w.N / (ms * 1e-3) / 1e9
     desc = w.describe()
     if w.noise_kind == I.NOISE_STUDENT_T3:
-        desc += " [t3 drawn as spherical pairs: elements 2m, 2m+1 share one radius]"
+        desc += " [elements 2m, 2m+1 of the t3 noise share one radius: each is t3, the pair is uncorrelated, not independent]"
     if algorithm == "ecsgd":
         desc += " [centralized error-compensated SGD: ds_ecsgd_step]"
     fused = info.path == B.DS_PATH_FUSED
