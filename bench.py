@@ -50,8 +50,8 @@ def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) ->
 # DRAM bytes per update of the dominant kernel from one ncu capture of a small case
 # (dram__bytes_read.sum + dram__bytes_write.sum over one launch of 67,108,864 updates,
 # scaled per update), valid for the kernel sources whose digest is recorded beside it.
-NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59477e9 / 67108864,
-               "sources_sha256": "70a26dd3c0391f05e2eb5a296d21be63deab540aeaecb024c6077ee900865e51"}
+NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59492e9 / 67108864,
+               "sources_sha256": "529d1acaf209c3ad12b0a7eb07f2e3aa9ed88d4bfa232cff9d6bff88a590e09a"}
 KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
 
 
