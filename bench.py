@@ -51,7 +51,7 @@ def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) ->
 # (dram__bytes_read.sum + dram__bytes_write.sum over one launch of 67,108,864 updates,
 # scaled per update), valid for the kernel sources whose digest is recorded beside it.
 NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59492e9 / 67108864,
-               "sources_sha256": "529d1acaf209c3ad12b0a7eb07f2e3aa9ed88d4bfa232cff9d6bff88a590e09a"}
+               "sources_sha256": "252801dbc2b9f3284fbd130e016f08d5566c7fac88e4bd336e46b12872d4fede"}
 KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
 
 

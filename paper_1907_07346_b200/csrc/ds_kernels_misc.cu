@@ -227,7 +227,7 @@ __global__ void __launch_bounds__(256) ds_math_selftest_kernel(unsigned long lon
         const float t = __fmul_rn(-2.0f, lg.x);
         if (__float_as_uint(sqrt_of_minus2log(t)) != __float_as_uint(__fsqrt_rn(t))) ++bad_sqrt;
         const float2 q = t3_radius_sq_x2(j, j2);
-        if (__float_as_uint(sqrt_one_correction(q.x)) != __float_as_uint(__fsqrt_rn(q.x))) ++bad_t3;
+        if (__float_as_uint(sqrt_of_minus2log(q.x)) != __float_as_uint(__fsqrt_rn(q.x))) ++bad_t3;
     }
     if (bad_log) atomicAdd(&counts[0], (unsigned long long)bad_log);
     if (bad_sqrt) atomicAdd(&counts[1], (unsigned long long)bad_sqrt);

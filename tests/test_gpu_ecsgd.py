@@ -62,7 +62,9 @@ def run_ecsgd(env, graph, N, kind, bits, chunk, noise, steps=1, seed=5, sigma=0.
 
 COMPS = [(I.COMP_SIGN1_L1, 1, 128), (I.COMP_SIGN1_L1, 1, 0), (I.COMP_UNIFORM_STOCH_MAXABS, 2, 256),
          (I.COMP_UNIFORM_STOCH_MAXABS, 4, 512), (I.COMP_UNIFORM_STOCH_MAXABS, 4, 0),
-         (I.COMP_UNIFORM_STOCH_MAXABS, 8, 64), (I.COMP_UNIFORM_NEAREST_L2, 4, 96), (I.COMP_IDENTITY, 32, 0)]
+         (I.COMP_UNIFORM_STOCH_MAXABS, 8, 64), (I.COMP_UNIFORM_NEAREST_L2, 4, 96), (I.COMP_IDENTITY, 32, 0),
+         # the paper's codec at its own granularity (one norm per tensor) and on chunks several warps share
+         (I.COMP_UNIFORM_NEAREST_L2, 4, 0), (I.COMP_UNIFORM_NEAREST_L2, 2, 1024)]
 
 
 @pytest.mark.parametrize("path", [0, 2])

@@ -15,6 +15,8 @@ CASES = {
     "chunk512_4bit_ring16": (I.ring(16), 512 * 5 + 40, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_GAUSS),
     "chunk1024_sign_torus": (I.torus(4, 8), 1024 * 3 + 130, I.COMP_SIGN1_L1, 1, 1024, I.NOISE_STUDENT_T3),
     "chunk256_norm2_exp16": (I.exponential(16), 256 * 9 + 8, I.COMP_UNIFORM_NEAREST_L2, 2, 256, I.NOISE_NONE),
+    # one norm per tensor: five launches per iteration in the graph
+    "per_tensor_norm4_ring8": (I.ring(8), 512 * 7 + 9, I.COMP_UNIFORM_NEAREST_L2, 4, 0, I.NOISE_GAUSS),
 }
 
 
