@@ -51,7 +51,7 @@ def algorithmic_bytes_per_update(w: I.Workload, given_gradient: bool = False) ->
 # (dram__bytes_read.sum + dram__bytes_write.sum over one launch of 67,108,864 updates,
 # scaled per update), valid for the kernel sources whose digest is recorded beside it.
 NCU_TRAFFIC = {"kernel": "ds_fused_tma_kernel", "workload": "cfg3", "bytes_per_update": 1.59492e9 / 67108864,
-               "sources_sha256": "252801dbc2b9f3284fbd130e016f08d5566c7fac88e4bd336e46b12872d4fede"}
+               "sources_sha256": "4cdbfdb9daee43c8ce108f76b785a0449b103167ccdcf77e02b0c4b9457180cc"}
 KERNEL_SOURCES = ["ds_fused_tma_kernel.cuh", "ds_column_kernel.cuh", "ds_device.cuh", "ds_internal.h"]
 
 
@@ -215,10 +215,14 @@ KERNEL_OF = {"cfg1": "ds_column_kernel (reduce) + ds_finalize_scales_kernel + ds
 
 
 def other_workload_line(torch, B, name: str, steps: int, dev, local_rank: int, peak: float,
-                        algorithm: str = "deepsqueeze", shared=None):
+                        algorithm: str = "deepsqueeze", shared=None, noise_kind=None):
     """One secondary timing line: `steps` device-timed steps of another workload (or of
-    centralized error-compensated SGD on the headline shape) on its default path."""
+    centralized error-compensated SGD on the headline shape) on its default path.
+    noise_kind: the workload with another gradient-noise kind."""
     w = I.WORKLOADS[name]
+    if noise_kind is not None:
+        w = w.with_size(w.N)
+        w.noise_kind = noise_kind
     ld = I.row_pitch(w.N)
     g = w.build_graph()
     stream = torch.cuda.current_stream(dev)
@@ -258,6 +262,8 @@ def other_workload_line(torch, B, name: str, steps: int, dev, local_rank: int, p
     kernel = (KERNEL_OF.get(name, "?") if fused else "not the TMA-staged path")
     if algorithm == "ecsgd":
         kernel = "ds_fused_tma_kernel (error-compensated SGD instantiation)"
+    if noise_kind == I.NOISE_STUDENT_T3_IID and name == "cfg4":
+        kernel = "ds_fused_tma_kernel (one node per warp, 1024 threads: the two-nodes-per-warp kernel does not take this noise)"
     line = {"workload": desc, "kernel": kernel, "steps": steps, "ms_per_step": ms,
             "updates_per_s": w.n * w.N / (ms * 1e-3), "algorithmic_bytes_per_update": b_alg,
             "achieved": achieved, "frac": achieved / peak,
@@ -517,6 +523,11 @@ def main():
         for name in ("cfg2", "cfg4", "cfg5"):
             others.append(other_workload_line(torch, B, name, args.other_steps, dev, local_rank, peak))
             torch.cuda.empty_cache()
+        # cfg4 with independent Student-t(3) coordinates (four normals per element): the reading of
+        # "Student-t(3) gradient noise" that is bound by the instruction stream instead of memory
+        others.append(other_workload_line(torch, B, "cfg4", max(10, args.other_steps // 5), dev, local_rank, peak,
+                                          noise_kind=I.NOISE_STUDENT_T3_IID))
+        torch.cuda.empty_cache()
 
     base = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -108,9 +108,16 @@ typedef struct {
 typedef enum {
     DS_NOISE_NONE = 0,
     DS_NOISE_GAUSS = 1,         /* standard normal (Box-Muller) */
-    DS_NOISE_STUDENT_T3 = 2     /* Student t, 3 degrees of freedom, not re-normalised: consecutive
+    DS_NOISE_STUDENT_T3 = 2,    /* Student t, 3 degrees of freedom, not re-normalised: consecutive
                                    elements (2m, 2m+1) form a spherical bivariate t(3) pair
                                    (each exactly t(3), uncorrelated, sharing one radius) */
+    DS_NOISE_STUDENT_T3_IID = 3 /* the same marginal law with INDEPENDENT coordinates, by the textbook
+                                   construction Z0 / sqrt((Z1^2 + Z2^2 + Z3^2) / 3): one Philox block
+                                   and four normals per element -- about three times the arithmetic
+                                   of the pairs, so steps with it are bound by the instruction
+                                   stream, not by memory.  Not taken by ds_run_resident
+                                   (DS_ERR_UNSUPPORTED) nor by the two-nodes-per-warp kernel (such
+                                   shapes run on the one-node-per-warp kernel) */
 } ds_noise_kind;
 
 typedef struct {

@@ -194,7 +194,7 @@ float oracle_t3_radius_u24(uint32_t j)
     return sqrtf(3.0f * E);
 }
 
-enum { NOISE_NONE = 0, NOISE_GAUSS = 1, NOISE_STUDENT_T3 = 2 };
+enum { NOISE_NONE = 0, NOISE_GAUSS = 1, NOISE_STUDENT_T3 = 2, NOISE_STUDENT_T3_IID = 3 };
 
 /* Unit noise z for element k of a node (before the factor sigma).
  * Block k/4 of the noise stream yields the elements 4m..4m+3: words (0,1) ->
@@ -204,12 +204,27 @@ enum { NOISE_NONE = 0, NOISE_GAUSS = 1, NOISE_STUDENT_T3 = 2 };
  *   GAUSS:      rho = sqrt(-2 ln u1)              (Box-Muller: two independent normals)
  *   STUDENT_T3: rho = sqrt(3 (u1^(-2/3) - 1))     (a spherical bivariate t(3) pair:
  *               each element is exactly t(3)-distributed; the two elements of a
- *               pair are uncorrelated but share their radius; pairs are independent). */
+ *               pair are uncorrelated but share their radius; pairs are independent).
+ * STUDENT_T3_IID: independent t(3) coordinates by the textbook construction
+ *   t = Z0 / sqrt((Z1^2 + Z2^2 + Z3^2) / 3) from four independent normals: element
+ *   k owns block k of the noise stream, (w0, w1) -> Z0, Z1 and (w2, w3) -> Z2, Z3
+ *   by Box-Muller as above, q = fma(Z3, Z3, fma(Z2, Z2, Z1 Z1)),
+ *   t = Z0 / sqrt(q / 3) (t = 0 if q = 0). */
 float oracle_noise_elem(int kind, uint64_t seed, uint32_t node, uint64_t step,
                         int64_t k)
 {
     uint32_t w[4];
     float z0, z1;
+    if (kind == NOISE_STUDENT_T3_IID) {
+        float z2, z3;
+        philox_block(seed, node, step, STREAM_NOISE, (uint32_t)k, w);
+        box_muller(w[0], w[1], &z0, &z1);
+        box_muller(w[2], w[3], &z2, &z3);
+        float q = fmaf(z3, z3, fmaf(z2, z2, z1 * z1));
+        if (q == 0.0f) return 0.0f;
+        float third = q / 3.0f;
+        return z0 / sqrtf(third);
+    }
     if (kind == NOISE_GAUSS || kind == NOISE_STUDENT_T3) {
         philox_block(seed, node, step, STREAM_NOISE, (uint32_t)(k >> 2), w);
         int pair = (int)((k >> 1) & 1);

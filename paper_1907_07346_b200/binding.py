@@ -21,7 +21,7 @@ DS_OK = 0
  DS_ERR_TIMEOUT, DS_ERR_BOUNDS) = range(1, 13)
 
 DS_COMP_IDENTITY, DS_COMP_SIGN1_L1, DS_COMP_UNIFORM_STOCH_MAXABS, DS_COMP_UNIFORM_NEAREST_L2 = 0, 1, 2, 3
-DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3 = 0, 1, 2
+DS_NOISE_NONE, DS_NOISE_GAUSS, DS_NOISE_STUDENT_T3, DS_NOISE_STUDENT_T3_IID = 0, 1, 2, 3
 DS_PATH_AUTO, DS_PATH_FUSED, DS_PATH_SPLIT, DS_PATH_FUSED_LDG = 0, 1, 2, 3
 DS_RUN_MAX_STEPS = 4096
 DS_RESIDENT_MAX_STEPS = 1024

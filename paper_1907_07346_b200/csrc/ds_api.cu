@@ -18,6 +18,9 @@ using namespace ds;
 
 namespace {
 
+// ds_noise_kind -> the kernels' NOISE_* value (GRAD_GIVEN sits between them)
+inline int noise_template_of(int32_t noise) { return noise == DS_NOISE_STUDENT_T3_IID ? (int)NOISE_T3I : (int)noise; }
+
 constexpr size_t kAlign = 256;
 constexpr int64_t kPerNodeTile = 512;   // tile width when one scale covers a node
 constexpr int kMaxSmem = 227 * 1024;
@@ -553,7 +556,7 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
         // (16 elements per lane, at most 512 threads), else two kernels
         const bool ecsgd_fused = ecsgd && ctx->path_req != DS_PATH_SPLIT && ctx->path_req != DS_PATH_FUSED_LDG &&
                                  ctx->tma.ok && ctx->tma.elems_per_lane == 16 && ctx->tma.block.x <= 512;
-        const int kind = ecsgd ? 0 : fused_kind(ctx, grad_kind == GRAD_GIVEN);
+        const int kind = ecsgd ? 0 : fused_kind(ctx, grad_kind == GRAD_GIVEN || grad_kind == NOISE_T3I);
         if (ecsgd_fused) {
             p.ecsgd = 0;          // the fused kernel is its own instantiation; the flag is for the two-kernel path
             p.warps_per_group = ctx->tma.warps_per_group;
@@ -597,8 +600,8 @@ static ds_status run_step(ds_ctx* ctx, float* x, float* delta, const float* a, c
 ds_status ds_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const ds_hparams* hp,
                   uint64_t seed, uint64_t step, void* cuda_stream) {
     if (!ctx || !x || !delta || !gp || !hp || !gp->a || !gp->c) return DS_ERR_NULL;
-    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
-    return run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, gp->noise, hp, seed, step, cuda_stream);
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3_IID) return DS_ERR_ARG;
+    return run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, noise_template_of(gp->noise), hp, seed, step, cuda_stream);
 }
 
 ds_status ds_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, const ds_hparams* hp,
@@ -610,9 +613,9 @@ ds_status ds_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, const d
 ds_status ds_ecsgd_step(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, float gamma,
                         uint64_t seed, uint64_t step, void* cuda_stream) {
     if (!ctx || !x || !delta || !gp || !gp->a || !gp->c) return DS_ERR_NULL;
-    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3_IID) return DS_ERR_ARG;
     const ds_hparams hp = {gamma, 0.0f};
-    return run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, gp->noise, &hp, seed, step, cuda_stream, 0, -1, true);
+    return run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, noise_template_of(gp->noise), &hp, seed, step, cuda_stream, 0, -1, true);
 }
 
 ds_status ds_ecsgd_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, float gamma,
@@ -625,7 +628,7 @@ ds_status ds_ecsgd_step_g(ds_ctx* ctx, float* x, float* delta, const float* g, f
 ds_status ds_run(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const float* gammas,
                  const float* etas, int32_t T, uint64_t seed, uint64_t step0, void* cuda_stream) {
     if (!ctx || !x || !delta || !gp || !gp->a || !gp->c || !gammas || !etas) return DS_ERR_NULL;
-    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3_IID) return DS_ERR_ARG;
     if (T < 1 || T > DS_RUN_MAX_STEPS) return DS_ERR_ARG;
     if (step0 >= ((uint64_t)1 << 56) || step0 + (uint64_t)T > ((uint64_t)1 << 56)) return DS_ERR_ARG;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
@@ -645,7 +648,7 @@ ds_status ds_run(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, 
     ds_status st = DS_OK;
     for (int32_t t = 0; t < T && st == DS_OK; ++t) {
         const ds_hparams hp = {gammas[t], etas[t]};
-        st = run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, gp->noise, &hp, seed, step0 + (uint64_t)t,
+        st = run_step(ctx, x, delta, gp->a, gp->c, gp->sigma, noise_template_of(gp->noise), &hp, seed, step0 + (uint64_t)t,
                       ctx->capture_stream);
     }
     cudaGraph_t graph = nullptr;
@@ -690,13 +693,13 @@ ds_status ds_run(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, 
 ds_status ds_run_resident(ds_ctx* ctx, float* x, float* delta, const ds_grad_params* gp, const float* gammas,
                           const float* etas, int32_t T, uint64_t seed, uint64_t step0, void* cuda_stream) {
     if (!ctx || !x || !delta || !gp || !gp->a || !gp->c || !gammas || !etas) return DS_ERR_NULL;
-    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3_IID) return DS_ERR_ARG;
     if (T < 1 || T > DS_RESIDENT_MAX_STEPS) return DS_ERR_ARG;
     if (step0 >= ((uint64_t)1 << 56) || step0 + (uint64_t)T > ((uint64_t)1 << 56)) return DS_ERR_ARG;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
                            reinterpret_cast<uintptr_t>(gp->a) | reinterpret_cast<uintptr_t>(gp->c);
     if ((bits % 16) != 0) return DS_ERR_ALIGN;
-    if (!resident_shape(ctx->n, ctx->sh)) return DS_ERR_UNSUPPORTED;
+    if (!resident_shape(ctx->n, ctx->sh) || gp->noise == DS_NOISE_STUDENT_T3_IID) return DS_ERR_UNSUPPORTED;
     if (resident_smem_layout(ctx->n, ctx->nnz).total > (size_t)kMaxSmem) return DS_ERR_UNSUPPORTED;
 
     static_assert(DS_RESIDENT_MAX_STEPS == kResidentMaxSteps, "header and kernel disagree");
@@ -760,7 +763,7 @@ ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const floa
     if (!ctx || !x_host || !delta_host || !a_host || !c_host || !hp || !dev_x || !dev_delta ||
         !dev_a || !dev_c)
         return DS_ERR_NULL;
-    if (noise < DS_NOISE_NONE || noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    if (noise < DS_NOISE_NONE || noise > DS_NOISE_STUDENT_T3_IID) return DS_ERR_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t pitch = (size_t)ctx->ld * sizeof(float);
     const size_t bytes = (size_t)ctx->n * pitch;
@@ -778,7 +781,7 @@ ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const floa
         if (e == cudaSuccess) e = cudaMemcpyAsync(dev_a, a_host, bytes, cudaMemcpyHostToDevice, stream);
         if (e == cudaSuccess) e = cudaMemcpyAsync(dev_c, c_host, bytes, cudaMemcpyHostToDevice, stream);
         if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
-        const ds_status st = run_step(ctx, dev_x, dev_delta, dev_a, dev_c, sigma, noise, hp, seed, step, cuda_stream);
+        const ds_status st = run_step(ctx, dev_x, dev_delta, dev_a, dev_c, sigma, noise_template_of(noise), hp, seed, step, cuda_stream);
         if (st != DS_OK) return st;
         e = cudaMemcpyAsync(x_host, dev_x, bytes, cudaMemcpyDeviceToHost, stream);
         if (e == cudaSuccess) e = cudaMemcpyAsync(delta_host, dev_delta, bytes, cudaMemcpyDeviceToHost, stream);
@@ -806,7 +809,7 @@ ds_status ds_step_host(ds_ctx* ctx, float* x_host, float* delta_host, const floa
         if (e == cudaSuccess) e = cudaEventRecord(ctx->pipe_event[2 * sidx], s_in);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(s_run, ctx->pipe_event[2 * sidx], 0);
         if (e != cudaSuccess) break;
-        failed = run_step(ctx, dev_x, dev_delta, dev_a, dev_c, sigma, noise, hp, seed, step, s_run, t0, t1);
+        failed = run_step(ctx, dev_x, dev_delta, dev_a, dev_c, sigma, noise_template_of(noise), hp, seed, step, s_run, t0, t1);
         if (failed != DS_OK) break;
         e = cudaEventRecord(ctx->pipe_event[2 * sidx + 1], s_run);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, ctx->pipe_event[2 * sidx + 1], 0);
@@ -896,9 +899,9 @@ ds_status ds_noise(float* out, int32_t n, int64_t N, int64_t ld_out, int32_t whi
                    uint64_t seed, uint64_t step, void* cuda_stream) {
     if (!out) return DS_ERR_NULL;
     if (n < 1 || N < 1 || N >= ((int64_t)1 << 31) || ld_out < N || which < 0 || which > 1 ||
-        noise < DS_NOISE_NONE || noise > DS_NOISE_STUDENT_T3 || step >= ((uint64_t)1 << 56))
+        noise < DS_NOISE_NONE || noise > DS_NOISE_STUDENT_T3_IID || step >= ((uint64_t)1 << 56))
         return DS_ERR_ARG;
-    const cudaError_t e = launch_noise_kernel(out, n, N, ld_out, which, noise, make_rng_step(seed, step),
+    const cudaError_t e = launch_noise_kernel(out, n, N, ld_out, which, noise_template_of(noise), make_rng_step(seed, step),
                                               static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) { (void)cudaGetLastError(); return DS_ERR_CUDA; }
     return DS_OK;

@@ -538,6 +538,7 @@ cudaError_t launch_code(const LaunchShape& sh, const StepParams& p, cudaStream_t
     DS_CASE(NOISE_NONE, 4) DS_CASE(NOISE_NONE, 8) DS_CASE(NOISE_NONE, 16)
     DS_CASE(NOISE_GAUSS, 4) DS_CASE(NOISE_GAUSS, 8) DS_CASE(NOISE_GAUSS, 16)
     DS_CASE(NOISE_T3, 4) DS_CASE(NOISE_T3, 8) DS_CASE(NOISE_T3, 16)
+    DS_CASE(NOISE_T3I, 4) DS_CASE(NOISE_T3I, 8) DS_CASE(NOISE_T3I, 16)
     DS_CASE(GRAD_GIVEN, 4) DS_CASE(GRAD_GIVEN, 8) DS_CASE(GRAD_GIVEN, 16)
 #undef DS_CASE
     return cudaErrorInvalidValue;

@@ -570,7 +570,7 @@ cudaError_t launch_tma_ecsgd_code(const LaunchShape& sh, const StepParams& p, cu
         kern<<<sh.grid, sh.block, sh.smem, stream>>>(p); \
         return cudaGetLastError(); \
     }
-    DS_TMA_EC_CASE(NOISE_NONE) DS_TMA_EC_CASE(NOISE_GAUSS) DS_TMA_EC_CASE(NOISE_T3) DS_TMA_EC_CASE(GRAD_GIVEN)
+    DS_TMA_EC_CASE(NOISE_NONE) DS_TMA_EC_CASE(NOISE_GAUSS) DS_TMA_EC_CASE(NOISE_T3) DS_TMA_EC_CASE(NOISE_T3I) DS_TMA_EC_CASE(GRAD_GIVEN)
 #undef DS_TMA_EC_CASE
     return cudaErrorInvalidValue;
 }
@@ -582,6 +582,7 @@ cudaError_t launch_tma_code(const LaunchShape& sh, const StepParams& p, cudaStre
     DS_TMA_CASE(NOISE_NONE, 4) DS_TMA_CASE(NOISE_NONE, 8) DS_TMA_CASE(NOISE_NONE, 16)
     DS_TMA_CASE(NOISE_GAUSS, 4) DS_TMA_CASE(NOISE_GAUSS, 8) DS_TMA_CASE(NOISE_GAUSS, 16)
     DS_TMA_CASE(NOISE_T3, 4) DS_TMA_CASE(NOISE_T3, 8) DS_TMA_CASE(NOISE_T3, 16)
+    DS_TMA_CASE(NOISE_T3I, 4) DS_TMA_CASE(NOISE_T3I, 8) DS_TMA_CASE(NOISE_T3I, 16)
     DS_TMA_CASE(GRAD_GIVEN, 4) DS_TMA_CASE(GRAD_GIVEN, 8) DS_TMA_CASE(GRAD_GIVEN, 16)
 #undef DS_TMA_CASE
     return cudaErrorInvalidValue;

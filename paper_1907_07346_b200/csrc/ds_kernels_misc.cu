@@ -177,6 +177,7 @@ __global__ void __launch_bounds__(256) ds_noise_kernel(float* out, int32_t n, in
         if (which == 1) z = rnd24x4(rs, (uint32_t)node, k);
         else if (noise == NOISE_GAUSS) z = noise4<NOISE_GAUSS>(rs, (uint32_t)node, k);
         else if (noise == NOISE_T3) z = noise4<NOISE_T3>(rs, (uint32_t)node, k);
+        else if (noise == NOISE_T3I) z = noise4<NOISE_T3I>(rs, (uint32_t)node, k);
         else z = make_float4(0.f, 0.f, 0.f, 0.f);
         const float zv[4] = {z.x, z.y, z.z, z.w};
         float* o = out + (size_t)node * (size_t)ld + (size_t)(4 * f);

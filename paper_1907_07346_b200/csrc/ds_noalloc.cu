@@ -66,7 +66,7 @@ extern "C" ds_status ds_node_scales_noalloc(float* scales_out, const float* x, c
                                             uint64_t step, void* cuda_stream) {
     if (!scales_out || !x || !delta || !gp || !gp->a || !gp->c) return DS_ERR_NULL;
     if (n < 1 || N < 1 || N >= ((int64_t)1 << 31) || ld < N || step >= ((uint64_t)1 << 56)) return DS_ERR_ARG;
-    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3) return DS_ERR_ARG;
+    if (gp->noise < DS_NOISE_NONE || gp->noise > DS_NOISE_STUDENT_T3_IID) return DS_ERR_ARG;
     if (comp_kind != DS_COMP_SIGN1_L1 && comp_kind != DS_COMP_UNIFORM_STOCH_MAXABS) return DS_ERR_ARG;
     if ((ld % 4) != 0) return DS_ERR_ALIGN;
     const uintptr_t bits = reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(delta) |
@@ -111,7 +111,7 @@ extern "C" ds_status ds_node_scales_noalloc(float* scales_out, const float* x, c
 
     LaunchShape sh;
     sh.code = code;
-    sh.noise = gp->noise;
+    sh.noise = (gp->noise == DS_NOISE_STUDENT_T3_IID) ? (int)NOISE_T3I : (int)gp->noise;
     sh.elems_per_lane = 16;
     sh.mode = MODE_REDUCE;
     sh.grid = dim3((unsigned)tiles, (unsigned)((n + npb - 1) / npb));

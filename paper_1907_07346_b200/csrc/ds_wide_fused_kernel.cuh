@@ -352,6 +352,7 @@ cudaError_t launch_wide_code(const LaunchShape& sh, const StepParams& p, cudaStr
     DS_WIDE_CASE(NOISE_NONE, 4) DS_WIDE_CASE(NOISE_NONE, 8) DS_WIDE_CASE(NOISE_NONE, 16)
     DS_WIDE_CASE(NOISE_GAUSS, 4) DS_WIDE_CASE(NOISE_GAUSS, 8) DS_WIDE_CASE(NOISE_GAUSS, 16)
     DS_WIDE_CASE(NOISE_T3, 4) DS_WIDE_CASE(NOISE_T3, 8) DS_WIDE_CASE(NOISE_T3, 16)
+    DS_WIDE_CASE(NOISE_T3I, 4) DS_WIDE_CASE(NOISE_T3I, 8) DS_WIDE_CASE(NOISE_T3I, 16)
     DS_WIDE_CASE(GRAD_GIVEN, 4) DS_WIDE_CASE(GRAD_GIVEN, 8) DS_WIDE_CASE(GRAD_GIVEN, 16)
 #undef DS_WIDE_CASE
     return cudaErrorInvalidValue;

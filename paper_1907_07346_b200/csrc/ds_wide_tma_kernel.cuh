@@ -489,6 +489,7 @@ cudaError_t launch_wide_tma_code(const LaunchShape& sh, const StepParams& p, cud
     DS_WT_CASE(NOISE_NONE, 8) DS_WT_CASE(NOISE_NONE, 16)
     DS_WT_CASE(NOISE_GAUSS, 8) DS_WT_CASE(NOISE_GAUSS, 16)
     DS_WT_CASE(NOISE_T3, 8) DS_WT_CASE(NOISE_T3, 16)
+    DS_WT_CASE(NOISE_T3I, 8) DS_WT_CASE(NOISE_T3I, 16)
     DS_WT_CASE(GRAD_GIVEN, 8) DS_WT_CASE(GRAD_GIVEN, 16)
 #undef DS_WT_CASE
     return cudaErrorInvalidValue;

@@ -26,6 +26,7 @@ COMP_UNIFORM_NEAREST_L2 = 3
 NOISE_NONE = 0
 NOISE_GAUSS = 1
 NOISE_STUDENT_T3 = 2
+NOISE_STUDENT_T3_IID = 3
 
 
 @dataclass
@@ -148,7 +149,8 @@ class Workload:
                 COMP_UNIFORM_STOCH_MAXABS: f"{self.bits}-bit uniform stochastic max-abs",
                 COMP_UNIFORM_NEAREST_L2: f"{self.bits}-bit nearest-level norm-matched"}[self.comp_kind]
         chunk = f"chunk {self.chunk}" if self.chunk else "per-node scale"
-        noise = {NOISE_NONE: "none", NOISE_GAUSS: "gauss", NOISE_STUDENT_T3: "student-t3(spherical pairs)"}[self.noise_kind]
+        noise = {NOISE_NONE: "none", NOISE_GAUSS: "gauss", NOISE_STUDENT_T3: "student-t3(spherical pairs)",
+                 NOISE_STUDENT_T3_IID: "student-t3(independent coordinates)"}[self.noise_kind]
         return (f"{self.name}: n={self.n} {self.graph} N={self.N} {comp} {chunk} "
                 f"noise={noise} sigma={self.sigma} gamma={self.gamma} eta={self.eta}")
 

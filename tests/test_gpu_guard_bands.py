@@ -71,6 +71,7 @@ FAMILIES = {
     "fused_tma_given_gradient": (I.ring(16), I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_NONE, 1, "step_g"),
     "fused_tma_ecsgd": (I.complete(8), I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_GAUSS, 0, "ecsgd"),
     "pair_2bit_t3": (I.torus(4, 8), I.COMP_UNIFORM_STOCH_MAXABS, 2, 256, I.NOISE_STUDENT_T3, 1, "step"),
+    "fused_tma_32_warps_independent_t3": (I.torus(4, 8), I.COMP_UNIFORM_STOCH_MAXABS, 2, 256, I.NOISE_STUDENT_T3_IID, 1, "step"),
     "wide_tma_sign_chunk4096": (I.ring(8), I.COMP_SIGN1_L1, 1, 4096, I.NOISE_GAUSS, 1, "step"),
     "wide_tma_sign_64_nodes": (I.exponential(64), I.COMP_SIGN1_L1, 1, 1024, I.NOISE_GAUSS, 1, "step"),
     "wide_tma_4bit_40_nodes": (I.ring(40), I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, I.NOISE_GAUSS, 1, "step"),

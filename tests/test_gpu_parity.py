@@ -127,7 +127,7 @@ def run_case(env, graph, N, kind, bits, chunk, noise, path, steps=1, pad=None, s
 
 
 # ------------------------------------------------------------ raw streams
-@pytest.mark.parametrize("noise", [I.NOISE_GAUSS, I.NOISE_STUDENT_T3])
+@pytest.mark.parametrize("noise", [I.NOISE_GAUSS, I.NOISE_STUDENT_T3, I.NOISE_STUDENT_T3_IID])
 def test_noise_streams_bit_exact(env, noise):
     torch, orc, B = env
     n, N = 3, 4099
@@ -141,7 +141,7 @@ def test_noise_streams_bit_exact(env, noise):
     assert np.all(got[:, N:] == 0)
 
 
-@pytest.mark.parametrize("noise", [I.NOISE_GAUSS, I.NOISE_STUDENT_T3])
+@pytest.mark.parametrize("noise", [I.NOISE_GAUSS, I.NOISE_STUDENT_T3, I.NOISE_STUDENT_T3_IID])
 def test_noise_streams_bit_exact_two_million_elements(env, noise):
     """A long stretch of the stream (every exponent range of the radius occurs)."""
     torch, orc, B = env
@@ -198,10 +198,12 @@ def test_single_step_graphs(env, path, gname, comp, chunk):
 
 
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("noise", [I.NOISE_NONE, I.NOISE_STUDENT_T3])
+@pytest.mark.parametrize("noise", [I.NOISE_NONE, I.NOISE_STUDENT_T3, I.NOISE_STUDENT_T3_IID])
 def test_single_step_other_noise(env, path, noise):
     run_case(env, I.torus(4, 8), 256 * 6 + 40, I.COMP_UNIFORM_STOCH_MAXABS, 2, 256, noise, path)
     run_case(env, I.ring(8), 1024 * 2 + 7, I.COMP_SIGN1_L1, 1, 1024, noise, path)
+    run_case(env, I.ring(16), 512 * 3 + 5, I.COMP_UNIFORM_STOCH_MAXABS, 4, 512, noise, path, steps=2)
+    run_case(env, I.exponential(64), 1024 + 130, I.COMP_SIGN1_L1, 1, 1024, noise, path)
 
 
 @pytest.mark.parametrize("path", PATHS)

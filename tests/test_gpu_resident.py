@@ -59,11 +59,11 @@ def test_resident_rejects_what_it_cannot_hold(env):
     torch, orc, B = env
     dummy = torch.zeros((32, 1024), dtype=torch.float32, device="cuda")
 
-    def status_of(graph, N, kind, bits, chunk, T=2, step0=0):
+    def status_of(graph, N, kind, bits, chunk, T=2, step0=0, noise=I.NOISE_GAUSS):
         ds = B.DeepSqueeze(graph, N, N, kind, bits, chunk)
         t = dummy[:graph.n, :N].contiguous()
         try:
-            ds.ds_run_resident(t, t.clone(), t.clone(), t.clone(), 0.1, I.NOISE_GAUSS, [0.01] * T, [0.5] * T, 1, step0)
+            ds.ds_run_resident(t, t.clone(), t.clone(), t.clone(), 0.1, noise, [0.01] * T, [0.5] * T, 1, step0)
             ds.ds_sync()
             return B.DS_OK
         except B.DsError as err:
@@ -75,6 +75,7 @@ def test_resident_rejects_what_it_cannot_hold(env):
     assert status_of(I.ring(4), 1024, I.COMP_UNIFORM_STOCH_MAXABS, 4, 256) == B.DS_ERR_UNSUPPORTED     # chunk
     assert status_of(I.ring(4), 1024, I.COMP_UNIFORM_STOCH_MAXABS, 8, 512) == B.DS_ERR_UNSUPPORTED     # bits
     assert status_of(I.torus(4, 8), 1024, I.COMP_SIGN1_L1, 1, 512) == B.DS_ERR_UNSUPPORTED             # 32 nodes
+    assert status_of(I.ring(4), 1024, I.COMP_SIGN1_L1, 1, 512, noise=I.NOISE_STUDENT_T3_IID) == B.DS_ERR_UNSUPPORTED
     assert status_of(I.ring(4), 1024, I.COMP_SIGN1_L1, 1, 512, T=0) == B.DS_ERR_ARG
     assert status_of(I.ring(4), 1024, I.COMP_SIGN1_L1, 1, 512, T=B.DS_RESIDENT_MAX_STEPS + 1) == B.DS_ERR_ARG
     assert status_of(I.ring(4), 1024, I.COMP_SIGN1_L1, 1, 512, T=2, step0=(1 << 56) - 1) == B.DS_ERR_ARG

@@ -188,6 +188,45 @@ def test_student_t3_element_mapping():
         assert t[k] == np.float32(rho) * c[0] and t[k + 1] == np.float32(rho) * s[0]
 
 
+def test_student_t3_iid_distribution_and_independence():
+    """The independent-coordinates Student-t(3) noise: every element is t(3), and, unlike the
+    spherical pairs, neighbouring elements are INDEPENDENT: their squares are uncorrelated
+    (for a spherical pair they share the radius: the same statistic is far from zero there)."""
+    t = orc.noise_row(I.NOISE_STUDENT_T3_IID, 77, 1, 4, 0, 1 << 19).astype(np.float64)
+    assert stats.kstest(t[:200_000], "t", args=(3,)).pvalue > 1e-3
+    assert abs(np.median(np.abs(t)) - stats.t.ppf(0.75, 3)) < 1e-2
+    b = np.tanh(t) ** 2                     # bounded, so the heavy tails do not swamp the estimate
+    assert abs(np.corrcoef(b[0::2], b[1::2])[0, 1]) < 1e-2
+    assert abs(np.corrcoef(b[:-1], b[1:])[0, 1]) < 1e-2
+    pairs = np.tanh(orc.noise_row(I.NOISE_STUDENT_T3, 77, 1, 4, 0, 1 << 19).astype(np.float64)) ** 2
+    assert np.corrcoef(pairs[0::2], pairs[1::2])[0, 1] > 0.05       # the contrast: a shared radius
+
+
+def test_student_t3_iid_element_mapping():
+    """Element k owns block k of the noise stream: words (0,1) give Z0, Z1 and (2,3) give Z2, Z3
+    by Box-Muller (cosine first), and t = Z0 / sqrt((Z1^2 + Z2^2 + Z3^2)/3) -- rebuilt here from the
+    oracle's Philox, logarithm and sine/cosine with numpy binary32 arithmetic, and, as a looser
+    check of the formula itself, in binary64."""
+    seed, node, step, N = 4321, 1, 9, 48
+    t = orc.noise_row(I.NOISE_STUDENT_T3_IID, seed, node, step, 0, N)
+    f = np.float32
+    for k in range(N):
+        w = orc.philox(np.array([k, node, step, 0], dtype=np.uint32), np.array([seed, 0], dtype=np.uint32))
+        z = []
+        for a, b in ((0, 1), (2, 3)):
+            lg = orc.log_u24_array((int(w[a]) >> 8) + 1, 1)[0]
+            rho = np.sqrt(f(-2.0) * lg, dtype=np.float32)
+            c, s = orc.sincos_u24_array(int(w[b]) >> 8, 1)
+            z += [f(rho * c[0]), f(rho * s[0])]
+        z64 = [float(v) for v in z]
+        want64 = z64[0] / np.sqrt((z64[1] ** 2 + z64[2] ** 2 + z64[3] ** 2) / 3.0)
+        assert abs(float(t[k]) - want64) <= 1e-5 * max(1.0, abs(want64))
+        # binary32, operation by operation (the two fma's as exact binary64 products rounded once)
+        q = f(float(z[3]) * float(z[3]) + float(f(float(z[2]) * float(z[2]) + float(f(z[1] * z[1])))))
+        want = f(z[0] / np.sqrt(f(q / f(3.0)), dtype=np.float32))
+        assert t[k] == want, (k, t[k], want)
+
+
 def test_noise_none_is_zero():
     assert np.all(orc.noise_row(I.NOISE_NONE, 1, 0, 0, 0, 100) == 0)
 
