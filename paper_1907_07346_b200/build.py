@@ -54,7 +54,7 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     libdeepsqueeze_debug.so; load it with DEEPSQUEEZE_LIB=<that path>."""
     obj_dir, lib = (OBJ_DEBUG, LIB_DEBUG) if debug else (OBJ, LIB)
     extra = (["-Xptxas", "-v"] if verbose else []) + (["-DDS_DEBUG"] if debug else [])
-    if debug and not force and os.path.exists(lib):
+    if not force and os.path.exists(lib):
         # an up-to-date library is enough (its object files need not be kept)
         sources = set()
         for src in SOURCES:
