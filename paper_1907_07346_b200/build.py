@@ -18,7 +18,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdeepsqueeze.so")
-SOURCES = ["ds_api.cu", "ds_kernels_tma.cu", "ds_kernels_fused.cu", "ds_kernels_wide.cu", "ds_kernels_wide_tma.cu", "ds_kernels_compress.cu",
+SOURCES = ["ds_api.cu", "ds_kernels_tma.cu", "ds_kernels_tma_a.cu", "ds_kernels_tma_b.cu", "ds_kernels_tma_c.cu", "ds_kernels_fused.cu", "ds_kernels_wide.cu", "ds_kernels_wide_tma.cu", "ds_kernels_compress.cu",
            "ds_kernels_misc.cu", "ds_noalloc.cu", "ds_kernels_resident.cu", "ds_kernels_tma_pair.cu", "ds_kernels_tma_ecsgd.cu",
            "ds_kernels_wide_norm.cu", "ds_kernels_wide_tma_norm.cu", "ds_kernels_reduce_norm.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
