@@ -33,7 +33,7 @@ def _device_outputs(torch, ds):
     return codes, scales
 
 
-@pytest.mark.parametrize("name", ["cfg3", "cfg2", "cfg5", "cfg4"])
+@pytest.mark.parametrize("name", ["cfg3", "cfg2", "cfg5", "cfg4", "cfg3_l2"])
 def test_full_size_windows_and_paths(name):
     """Two free-running steps at the workload's full size on the default path (the kernel the
     benchmark times).  (1) 64 seeded random chunk columns plus windows at the start, in the
