@@ -33,6 +33,8 @@ def run(args):
     rows = [("none (D-PSGD)", I.COMP_IDENTITY, 32, 0), ("8-bit stochastic", I.COMP_UNIFORM_STOCH_MAXABS, 8, 512),
             ("4-bit stochastic", I.COMP_UNIFORM_STOCH_MAXABS, 4, 512), ("2-bit stochastic", I.COMP_UNIFORM_STOCH_MAXABS, 2, 512),
             ("4-bit nearest + norm", I.COMP_UNIFORM_NEAREST_L2, 4, 512), ("2-bit nearest + norm", I.COMP_UNIFORM_NEAREST_L2, 2, 512),
+            # the paper's own setting (Section 5): b bits per element and ONE norm per tensor
+            ("4-bit + norm per tensor", I.COMP_UNIFORM_NEAREST_L2, 4, 0), ("2-bit + norm per tensor", I.COMP_UNIFORM_NEAREST_L2, 2, 0),
             ("1-bit sign", I.COMP_SIGN1_L1, 1, 512)]
     out = []
     for name, kind, bits, chunk in rows:
