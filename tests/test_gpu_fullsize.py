@@ -152,3 +152,56 @@ def test_host_buffer_entry_point_pipelined():
     assert _rel(pinned[1].numpy()[:, :N], host[1][:, :N]) <= TOL
     assert np.all(pinned[0].numpy()[:, N:] == 3.0) and np.all(pinned[1].numpy()[:, N:] == 3.0)
     ds.close()
+
+
+@pytest.mark.parametrize("path", [0, 2], ids=["default-path", "two-kernels"])
+def test_longest_rows(path):
+    """Maximum size: N just below the 2^31 limit of the interface (two nodes, 4-bit codes, chunks of
+    512: 4,194,304 tiles per row, a ragged last one; 8.6 GB per array row, offsets beyond 2^32
+    bytes).  The state is drawn on the device; windows at the start, around the 2^30-th and 2^31-th
+    byte and element boundaries and at the very end of the rows are copied to the host and
+    compared with the oracle run on those columns (random streams indexed by the global column):
+    codes and floats bit for bit (max-abs scales), over two free-running steps."""
+    import torch
+    from oracle import oracle as orc
+    from paper_1907_07346_b200 import binding as B
+    from test_gpu_parity import assert_state_matches
+    g = I.complete(2)
+    chunk, bits, kind = 512, 4, I.COMP_UNIFORM_STOCH_MAXABS
+    N = (1 << 31) - 48                      # the interface takes N < 2^31; ld a multiple of 4
+    ld = N
+    M = (N + chunk - 1) // chunk
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(12345)
+    dev = []
+    for scale in (0.3, 0.05, None, 1.0):
+        t = torch.empty((g.n, ld), dtype=torch.float32, device="cuda")
+        for i in range(g.n):
+            if scale is None:
+                t[i].uniform_(0.5, 2.0, generator=gen)
+            else:
+                t[i].normal_(0.0, scale, generator=gen)
+        dev.append(t)
+    ds = B.DeepSqueeze(g, N, ld, kind, bits, chunk)
+    ds.ds_set_path(path)
+    if path == 0:
+        assert ds.ds_get_info().path == B.DS_PATH_FUSED and ds.ds_get_info().grid_blocks == 148
+    first_tiles = [0, (1 << 30) // 4 // chunk - 1, (1 << 30) // chunk - 1, (1 << 31) // 4 // chunk - 1, M // 2, M - 3]
+    windows = [(m * chunk, min(3 * chunk, N - m * chunk)) for m in first_tiles]
+    wstate = [[np.ascontiguousarray(t[:, k0:k0 + cols].cpu().numpy()) for t in dev] for k0, cols in windows]
+    sigma, gamma, eta, seed = 0.1, 0.01, 0.5, 4711
+    for step in range(2):
+        ds.ds_step(dev[0], dev[1], dev[2], dev[3], sigma, I.NOISE_GAUSS, gamma, eta, seed, step)
+        ds.ds_sync()
+        codes_d, scales_d = _device_outputs(torch, ds)
+        for (k0, cols), st in zip(windows, wstate):
+            cw, sw, _, _ = orc.step(g, kind, bits, chunk, st[0], st[1], st[2], st[3], cols, sigma, I.NOISE_GAUSS,
+                                    gamma, eta, seed, step, k_first=k0)
+            w0 = k0 * bits // 32
+            assert np.array_equal(codes_d[:, w0:w0 + cw.shape[1]].cpu().numpy().view(np.uint32), cw), (step, k0)
+            m0 = k0 // chunk
+            got_scales = scales_d[:, m0:m0 + sw.shape[1]].cpu().numpy().view(np.float32)
+            gx, gd = dev[0][:, k0:k0 + cols].cpu().numpy(), dev[1][:, k0:k0 + cols].cpu().numpy()
+            assert_state_matches(kind, cols, chunk, (gx, gd, got_scales), (st[0], st[1], sw), TOL, f"step {step} column {k0}")
+    assert bool(torch.isfinite(dev[0]).all()) and bool(torch.isfinite(dev[1]).all())
+    ds.close()
