@@ -86,8 +86,9 @@ typedef struct {
  *                                decodes to that norm: C = level[code] * ||v||_2 / ||level[code]||_2.
  *                                Deterministic and biased -- what error compensation is for.
  *                                One chunk = one "tensor"; chunk = 0 is the paper's granularity,
- *                                one norm for the node's whole vector (two more reduction
- *                                launches per step: the maximum, then the two sums of squares).
+ *                                one norm for the node's whole vector (five launches per step:
+ *                                maximum per tile, maximum per node, sums of squares per tile,
+ *                                norm per node, then the fused kernel with all three given).
  * chunk: elements per scale, a multiple of 32; 0 = one scale per node. */
 typedef enum {
     DS_COMP_IDENTITY = 0,
