@@ -275,6 +275,14 @@ def other_workload_line(torch, B, name: str, steps: int, dev, local_rank: int, p
     return line
 
 
+def guarded_line(what: str, fn, *a, **kw):
+    """A secondary line must never cost the headline: a failure becomes an entry that says so."""
+    try:
+        return fn(*a, **kw)
+    except Exception as err:            # noqa: BLE001 (reported, not swallowed)
+        return {"workload": what, "error": f"{type(err).__name__}: {err}"}
+
+
 def run_reference(args, w: I.Workload):
     """The reference arm: the CPU checker on a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
@@ -515,18 +523,18 @@ def main():
             and args.algorithm == "deepsqueeze" and not args.given_gradient and not args.elems_per_lane:
         others = []
         shared = (a, c, x, delta)
-        others.append(other_workload_line(torch, B, "cfg3", args.other_steps, dev, local_rank, peak, "ecsgd", shared))
-        others.append(other_workload_line(torch, B, "cfg3_l2", args.other_steps, dev, local_rank, peak, shared=shared))
+        others.append(guarded_line("cfg3 ecsgd", other_workload_line, torch, B, "cfg3", args.other_steps, dev, local_rank, peak, "ecsgd", shared))
+        others.append(guarded_line("cfg3_l2", other_workload_line, torch, B, "cfg3_l2", args.other_steps, dev, local_rank, peak, shared=shared))
         ds.close()
         del shared, a, c, x, delta
         torch.cuda.empty_cache()
         for name in ("cfg2", "cfg4", "cfg5"):
-            others.append(other_workload_line(torch, B, name, args.other_steps, dev, local_rank, peak))
+            others.append(guarded_line(name, other_workload_line, torch, B, name, args.other_steps, dev, local_rank, peak))
             torch.cuda.empty_cache()
         # cfg4 with independent Student-t(3) coordinates (four normals per element): the reading of
         # "Student-t(3) gradient noise" that is bound by the instruction stream instead of memory
-        others.append(other_workload_line(torch, B, "cfg4", max(10, args.other_steps // 5), dev, local_rank, peak,
-                                          noise_kind=I.NOISE_STUDENT_T3_IID))
+        others.append(guarded_line("cfg4 independent t3", other_workload_line, torch, B, "cfg4",
+                                   max(10, args.other_steps // 5), dev, local_rank, peak, noise_kind=I.NOISE_STUDENT_T3_IID))
         torch.cuda.empty_cache()
 
     base = None
